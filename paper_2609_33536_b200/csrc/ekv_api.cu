@@ -9,6 +9,7 @@ int64_t g_decode_chunk_tokens = 0;
 int64_t g_decode_variant = 0;
 int64_t g_decode_merge_slices = 0;
 int64_t g_prefill_variant = 0;
+int64_t g_attn_out_f32 = 0;
 void *g_profile_ev[2] = {nullptr, nullptr};
 
 __global__ void validate_batch_kernel(const int32_t *block_table, const int32_t *seq_lens, const uint8_t *tags,
@@ -70,6 +71,11 @@ extern "C" int ekv_set_option(const char *name, int64_t value)
     if (!strcmp(name, "decode_merge_slices")) {
         if (value != 0 && value != 1 && value != 4 && value != 8) return EKV_ERR_INVALID_ARG;
         g_decode_merge_slices = value;
+        return EKV_OK;
+    }
+    if (!strcmp(name, "attn_out_f32")) {
+        if (value != 0 && value != 1) return EKV_ERR_INVALID_ARG;
+        g_attn_out_f32 = value;
         return EKV_OK;
     }
     if (!strcmp(name, "decode_variant")) {

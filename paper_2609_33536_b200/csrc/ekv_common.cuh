@@ -15,6 +15,7 @@ extern int64_t g_decode_chunk_tokens;   // option "decode_chunk_tokens"; 0 = aut
 extern int64_t g_prefill_variant;       // option "prefill_variant"; 0 = automatic (tcgen05 kernel at head_dim 128), 1 = mma.sync kernel
 extern void *g_profile_ev[2];           // ekv_set_profile_events: recorded around the main kernel of a call
 extern int64_t g_decode_merge_slices;   // option "decode_merge_slices"; 0 = automatic, else 1, 4 or 8
+extern int64_t g_attn_out_f32;          // option "attn_out_f32"; 1 = attention entry points store fp32 outputs (debug)
 extern int64_t g_decode_variant;        // option "decode_variant"; 0 / 3 = ring-staged kernel, 1 = page-stepped comparator
 int decode_chunk_tokens(int batch, int num_kv_heads, int max_seq_len);
 size_t decode_workspace_bytes(int batch, int num_q_heads, int num_kv_heads, int head_dim, int max_seq_len);

@@ -25,6 +25,7 @@
 #include "ekv_common.cuh"
 #include <math.h>
 #include <string.h>
+#include <atomic>
 
 namespace ekv {
 
@@ -46,6 +47,7 @@ struct DecodeParams {
     int batch, num_q_heads, num_kv_heads, group, max_blocks;
     int chunk_tokens, max_splits;
     float scale_log2;                   // sm_scale * log2(e)
+    int out_f32;                        // debug: `out` is float [batch][Hq][D] and receives the unrounded result
 };
 
 __device__ __forceinline__ bool m_run_is_empty(float m) { return m == -INFINITY; }
@@ -93,8 +95,10 @@ __global__ void __launch_bounds__(kDecodeThreads, 3) decode_page_kernel(DecodePa
     if (split >= (n_splits > 0 ? n_splits : 1)) return;
     const int h0 = g * G;                                         // first query head of the group
     if (L <= 0) {                                                 // empty request: zeros
-        for (int i = threadIdx.x; i < G * D; i += kDecodeThreads)
-            p.out[((int64_t)r * p.num_q_heads + h0) * D + i] = __float2bfloat16(0.f);
+        for (int i = threadIdx.x; i < G * D; i += kDecodeThreads) {
+            if (p.out_f32) ((float *)p.out)[((int64_t)r * p.num_q_heads + h0) * D + i] = 0.f;
+            else p.out[((int64_t)r * p.num_q_heads + h0) * D + i] = __float2bfloat16(0.f);
+        }
         return;
     }
     const int t0 = split * p.chunk_tokens;
@@ -333,7 +337,8 @@ __global__ void __launch_bounds__(kDecodeThreads, 3) decode_page_kernel(DecodePa
         const float val = acc / lsum;
         const int64_t row = (int64_t)r * p.num_q_heads + h0 + h;
         if (n_splits == 1) {
-            p.out[row * D + d] = __float2bfloat16(val);
+            if (p.out_f32) ((float *)p.out)[row * D + d] = val;
+            else p.out[row * D + d] = __float2bfloat16(val);
         } else {
             p.part_o[(row * p.max_splits + split) * D + d] = val;
             if (d == 0) p.part_lse[row * p.max_splits + split] = M + log2f(lsum);
@@ -532,8 +537,10 @@ __global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(D
     if (split >= (n_splits > 0 ? n_splits : 1)) return;
     const int h0 = g * G;
     if (L <= 0) {
-        for (int i = threadIdx.x; i < G * D; i += kDecodeThreads)
-            ((uint16_t *)p.out)[((int64_t)r * p.num_q_heads + h0) * D + i] = 0;
+        for (int i = threadIdx.x; i < G * D; i += kDecodeThreads) {
+            if (p.out_f32) ((float *)p.out)[((int64_t)r * p.num_q_heads + h0) * D + i] = 0.f;
+            else ((uint16_t *)p.out)[((int64_t)r * p.num_q_heads + h0) * D + i] = 0;
+        }
         return;
     }
     const int t0 = split * p.chunk_tokens;
@@ -832,7 +839,8 @@ __global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(D
         const float val = acc / lsum;
         const int64_t row = (int64_t)r * p.num_q_heads + h0 + h;
         if (n_splits == 1) {
-            ((uint16_t *)p.out)[row * D + d] = f32_to_16<F16>(val);
+            if (p.out_f32) ((float *)p.out)[row * D + d] = val;
+            else ((uint16_t *)p.out)[row * D + d] = f32_to_16<F16>(val);
         } else {
             p.part_o[(row * p.max_splits + split) * D + d] = val;
             if (d == 0) p.part_lse[row * p.max_splits + split] = M + log2f(lsum);
@@ -919,7 +927,8 @@ __global__ void __launch_bounds__(D * SG) decode_merge_kernel(DecodeParams p)
 #pragma unroll
         for (int g = 0; g < SG; ++g) { acc += sm_acc[g][threadIdx.x]; wsum += sm_w[g]; }
     }
-    ((uint16_t *)p.out)[(int64_t)row * D + threadIdx.x] = f32_to_16<F16>(acc / wsum);
+    if (p.out_f32) ((float *)p.out)[(int64_t)row * D + threadIdx.x] = acc / wsum;
+    else ((uint16_t *)p.out)[(int64_t)row * D + threadIdx.x] = f32_to_16<F16>(acc / wsum);
 }
 
 // Launch the merge kernel so that its launch latency overlaps the tail of the split kernel.
@@ -967,7 +976,7 @@ int decode_chunk_tokens(int batch, int num_kv_heads, int max_seq_len)
 size_t decode_workspace_bytes(int batch, int num_q_heads, int num_kv_heads, int head_dim, int max_seq_len)
 {
     const int chunk = decode_chunk_tokens(batch, num_kv_heads, max_seq_len);
-    const int64_t max_splits = (max_seq_len + chunk - 1) / chunk;
+    const int64_t max_splits = ((int64_t)max_seq_len + chunk - 1) / chunk;
     if (max_splits <= 1) return 0;
     const int64_t rows = (int64_t)batch * num_q_heads * max_splits;
     return (size_t)(rows * head_dim * 4 + (rows * 4 + 255) / 256 * 256);
@@ -1012,6 +1021,7 @@ static int decode_impl(const ekv_pool *pool, int32_t layer, const ekv_batch *bat
     p.chunk_tokens = decode_chunk_tokens(batch->batch, pool->num_kv_heads, max_seq_len);
     p.max_splits = max_seq_len > 0 ? (max_seq_len + p.chunk_tokens - 1) / p.chunk_tokens : 1;
     p.scale_log2 = sm_scale * 1.4426950408889634f;
+    p.out_f32 = g_attn_out_f32 ? 1 : 0;
     if (p.max_splits > 1) {
         const size_t need = decode_workspace_bytes(batch->batch, num_q_heads, pool->num_kv_heads, pool->head_dim, max_seq_len);
         if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) return EKV_ERR_WORKSPACE;
@@ -1148,22 +1158,21 @@ constexpr size_t kNoAllocScratchBytes = 16u << 20;      // 16 MiB, held by every
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
 
 constexpr int kMaxDevices = 64;
-static void *g_noalloc_scratch_ptr[kMaxDevices];          // device address of the array, per device
-static bool g_noalloc_scratch_ready[kMaxDevices];
+static std::atomic<void *> g_noalloc_scratch_ptr[kMaxDevices];   // device address of the array, per device; null = not asked yet
 
 // In host code `g_noalloc_scratch` is only a handle; the device address has to be asked for,
-// once per device, with that device current.
+// once per device, with that device current. Host threads that make their first calls at the
+// same time each ask and store the same answer (release / acquire on the slot).
 static int noalloc_scratch_address(void **ptr)
 {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return EKV_ERR_CUDA;
-    if (!g_noalloc_scratch_ready[dev]) {
-        void *p = nullptr;
+    void *p = g_noalloc_scratch_ptr[dev].load(std::memory_order_acquire);
+    if (!p) {
         if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || p == nullptr) return EKV_ERR_CUDA;
-        g_noalloc_scratch_ptr[dev] = p;
-        g_noalloc_scratch_ready[dev] = true;
+        g_noalloc_scratch_ptr[dev].store(p, std::memory_order_release);
     }
-    *ptr = g_noalloc_scratch_ptr[dev];
+    *ptr = p;
     return EKV_OK;
 }
 
@@ -1175,7 +1184,11 @@ extern "C" int ekv_attn_decode_noalloc(const ekv_pool *pool, int32_t layer, cons
                                        const void *q, void *out, int32_t num_q_heads, float sm_scale,
                                        int32_t max_seq_len, void *stream)
 {
-    if (!pool || !batch || num_q_heads <= 0) return EKV_ERR_INVALID_ARG;
+    int rc0 = check_pool(pool);
+    if (rc0) return rc0;
+    rc0 = check_batch(batch);
+    if (rc0) return rc0;
+    if (num_q_heads <= 0 || max_seq_len < 0) return EKV_ERR_INVALID_ARG;
     // Refuse, before touching the GPU, any shape whose partials would not fit the fixed array.
     const size_t need = ekv_attn_workspace_bytes(pool, batch->batch, num_q_heads, max_seq_len, 0);
     if (need > ekv::kNoAllocScratchBytes) return EKV_ERR_WORKSPACE;

@@ -32,6 +32,7 @@ struct PrefillParams {
     int group_rows;                    // rows a token takes in a tile: the group size rounded up to a power of two
     int q_tiles;                       // tiles per request: ceil(max_q_len / (64 / group_rows))
     float scale_log2;
+    int out_f32;                       // debug: `out` is float and receives the unrounded result
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -294,6 +295,12 @@ __global__ void __launch_bounds__(kPfThreads, 2) prefill_chunk_kernel(PrefillPar
         const int i = i0 + m / Gp, hl = m % Gp, h = g * G + hl;
         if (i >= C || hl >= G) continue;
         const float inv = l > 0.f ? 1.f / l : 0.f;
+        if (p.out_f32) {
+            float2 *dst = (float2 *)((float *)p.out + ((int64_t)(qs + i) * p.num_q_heads + h) * D);
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) dst[4 * nt + j] = make_float2(o[nt][2 * hf] * inv, o[nt][2 * hf + 1] * inv);
+            continue;
+        }
         uint32_t *dst = (uint32_t *)(p.out + ((int64_t)(qs + i) * p.num_q_heads + h) * D);
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
@@ -316,6 +323,7 @@ struct PrefillTcParams {
     int split_first, splits;     // used by the warp-specialised kernel only
     float *part;
     int *part_count;
+    int out_f32;
 };
 int launch_prefill_ws(const PrefillTcParams &p, int64_t ctas, int max_pages, int num_blocks, bool has_base, bool f16,
                       void *workspace, size_t workspace_bytes, cudaStream_t st);
@@ -369,6 +377,7 @@ extern "C" int ekv_attn_prefill_chunk(const ekv_pool *pool, int32_t layer, const
         const int tok_tc = 2 * (128 / Gp);                // two row tiles of 128 rows per CTA
         tp.q_tiles = (max_q_len + tok_tc - 1) / tok_tc;
         tp.scale_log2 = sm_scale * 1.4426950408889634f;
+        tp.out_f32 = g_attn_out_f32 ? 1 : 0;
         const int64_t n = (int64_t)batch->batch * pool->num_kv_heads * tp.q_tiles;
         if (n > 0x7fffffffLL) return EKV_ERR_UNSUPPORTED;
         return launch_prefill_ws(tp, n, max_pages, pool->num_blocks, batch->has_base != 0, pool->elem_type == EKV_FP16, workspace, workspace_bytes, (cudaStream_t)stream);
@@ -393,6 +402,7 @@ extern "C" int ekv_attn_prefill_chunk(const ekv_pool *pool, int32_t layer, const
     const int tok_m = kPfRows / Gp;
     p.q_tiles = (max_q_len + tok_m - 1) / tok_m;
     p.scale_log2 = sm_scale * 1.4426950408889634f;
+    p.out_f32 = g_attn_out_f32 ? 1 : 0;
     const int64_t ctas = (int64_t)batch->batch * pool->num_kv_heads * p.q_tiles;
     if (ctas > 0x7fffffffLL) return EKV_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)stream;

@@ -85,6 +85,7 @@ struct PrefillTcParams {
     int split_first, splits;
     float *part;                 // [unit - split_first][piece]: kWsPartFloats floats
     int *part_count;             // [unit - split_first], zero at launch
+    int out_f32;                 // debug: `out` is float and receives the unrounded result
 };
 
 __device__ __forceinline__ uint32_t ws_smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -111,7 +112,7 @@ __device__ __forceinline__ void ws_mbar_expect(uint32_t bar, uint32_t bytes)    
     if (bytes) asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
     else ws_mbar_arrive(bar);
 }
-// Tiled TMA copy (no multicast) of one box at element (x, y) into shared memory; completes on `bar`.
+// Tiled TMA copy of one box at element (x, y) into this CTA's shared memory; completes on `bar`.
 __device__ __forceinline__ void ws_tma_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
 {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -545,7 +546,16 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_ws_kernel(PrefillTcPara
                     uint32_t v[32];
                     ws_ld32(tmem_o + q * 32, v);
                     ws_wait_ld();
-                    if (row_ok) {
+                    if (row_ok && p.out_f32) {
+                        float *dstf = (float *)p.out + ((int64_t)(qs + row_i[w]) * p.num_q_heads + (g * G + row % Gp)) * kWsD + hf * kWsCols + q * 32;
+#pragma unroll
+                        for (int c4 = 0; c4 < 8; ++c4) {
+                            uint32_t ow[4];
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) ow[i] = __float_as_uint(__uint_as_float(v[4 * c4 + i]) * inv);
+                            st16B(dstf + 4 * c4, ow);
+                        }
+                    } else if (row_ok) {
 #pragma unroll
                         for (int c4 = 0; c4 < 4; ++c4) {
                             uint32_t ow[4];
@@ -637,7 +647,16 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_ws_kernel(PrefillTcPara
                                 }
                             }
                         }
-                        if (row_ok) {
+                        if (row_ok && p.out_f32) {
+                            float *dstf = (float *)p.out + ((int64_t)(qs + row_i[w]) * p.num_q_heads + (g * G + row % Gp)) * kWsD + hf * kWsCols + q * 32;
+#pragma unroll
+                            for (int c4 = 0; c4 < 8; ++c4) {
+                                uint32_t ow[4];
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) ow[i] = __float_as_uint(acc[4 * c4 + i] * inv);
+                                st16B(dstf + 4 * c4, ow);
+                            }
+                        } else if (row_ok) {
 #pragma unroll
                             for (int c4 = 0; c4 < 4; ++c4) {
                                 uint32_t ow[4];

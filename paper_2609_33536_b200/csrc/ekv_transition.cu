@@ -4,8 +4,10 @@
 // slabs of one (pair, layer, tensor): a slab is 16*D*2 bytes both as one member's
 // TARGET words and as the pair's packed BASE bytes, so every in-place hazard (the kept block is
 // source and destination) stays inside the CTA: all loads, one barrier, all stores.
-// The block table and tags are only read by the data kernel; a second, tiny kernel publishes
-// the new mapping afterwards, so a partially written state is never visible to later work.
+// The block table and tags are only read by the data CTAs; the new mapping is published after all
+// of them are done -- by the CTA that finishes last when the batch is small (one launch per
+// transition), by a second, tiny kernel when it is large -- so a partially written state is never
+// visible to later work.
 #include "ekv_common.cuh"
 #include <atomic>
 

@@ -8,8 +8,7 @@ import pytest
 import torch
 
 from paper_2609_33536_b200 import synth
-from gpu_util import require_gpu, upload_state, mixed_oracle_pool, gpu_decode, assert_attn_close, dev_i32, words
-from test_gpu_prefill import gpu_prefill
+from gpu_util import require_gpu, upload_state, mixed_oracle_pool, gpu_decode, gpu_prefill, assert_attn_close, dev_i32, words
 
 pytestmark = pytest.mark.gpu
 
@@ -26,7 +25,7 @@ def _decode_check(oracle, wl, chunk=0, what=""):
         got = gpu_decode(b, pool, batch, q, wl.num_q_heads, wl.sm_scale)
     finally:
         b.ekv_set_option("decode_chunk_tokens", 0)
-    return assert_attn_close(got, exp, what or wl.name)
+    return assert_attn_close(got, exp, what or wl.name, elem_type="fp16")
 
 
 @pytest.mark.parametrize("D", [64, 128])
@@ -82,7 +81,7 @@ def test_structured_path_fp16(oracle):
         out = torch.full(q.shape, float("nan"), dtype=q.dtype, device="cuda")
         b.ekv_attn_decode_structured(pool, 0, batch, bounds, q, out, wl.num_q_heads, wl.sm_scale, int(wl.seq_lens.max()), ws)
         torch.cuda.synchronize()
-        assert_attn_close(out.to(torch.float64).cpu().numpy(), exp, "fp16 structured")
+        assert_attn_close(out.to(torch.float64).cpu().numpy(), exp, "fp16 structured", elem_type="fp16")
     else:
         pytest.skip("generator did not produce a T-B-T batch")
 
@@ -97,7 +96,7 @@ def test_prefill_ragged_mixed(oracle, D, G):
     op, *_ = mixed_oracle_pool(oracle, wl)
     exp = oracle.attn_prefill_chunk(op, 0, wl.q_start, wl.q, wl.num_q_heads, wl.sm_scale)
     pool, batch, q = upload_state(b, op, wl.q)
-    assert_attn_close(gpu_prefill(b, pool, batch, q, wl), exp, f"fp16 prefill D{D} G{G}")
+    assert_attn_close(gpu_prefill(b, pool, batch, q, wl), exp, f"fp16 prefill D{D} G{G}", elem_type="fp16")
 
 
 def test_prefill_pieces_fp16(oracle):
@@ -107,7 +106,7 @@ def test_prefill_pieces_fp16(oracle):
     op, *_ = mixed_oracle_pool(oracle, wl)
     exp = oracle.attn_prefill_chunk(op, 0, wl.q_start, wl.q, wl.num_q_heads, wl.sm_scale)
     pool, batch, q = upload_state(b, op, wl.q)
-    assert_attn_close(gpu_prefill(b, pool, batch, q, wl, with_workspace=True), exp, "fp16 prefill pieces")
+    assert_attn_close(gpu_prefill(b, pool, batch, q, wl, with_workspace=True), exp, "fp16 prefill pieces", elem_type="fp16")
 
 
 def test_transitions_bit_exact_on_fp16_pool(oracle):

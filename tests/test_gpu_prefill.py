@@ -5,26 +5,9 @@ import pytest
 import torch
 
 from paper_2609_33536_b200 import synth
-from gpu_util import require_gpu, upload_state, mixed_oracle_pool, assert_attn_close
+from gpu_util import require_gpu, upload_state, mixed_oracle_pool, assert_attn_close, gpu_prefill
 
 pytestmark = pytest.mark.gpu
-
-
-def gpu_prefill(b, pool, batch, q, wl, layer=0, with_workspace=False):
-    """with_workspace: hand the call the workspace it asks for, which lets the tcgen05 kernel cut the
-    units of its last wave into pieces along the KV axis (merged by the piece that finishes last)."""
-    qs = torch.from_numpy(wl.q_start).cuda()
-    out = torch.full(q.shape, float("nan"), dtype=q.dtype, device="cuda")
-    chunk = np.diff(wl.q_start)
-    ws = None
-    if with_workspace:
-        ws = b.new_workspace(pool, len(wl.seq_lens), wl.num_q_heads, int(wl.seq_lens.max()), int(wl.q_start[-1]))
-        ws.fill_(0xA5)                                    # the call must not rely on what the workspace holds
-    b.ekv_attn_prefill_chunk(pool, layer, batch, qs, q, out, wl.num_q_heads, wl.sm_scale,
-                             int(wl.q_start[-1]), int(chunk.max()), int(wl.seq_lens.max()), ws)
-    torch.cuda.synchronize()
-    assert b.ekv_prefill_status() == 0, "a bounded wait inside the tensor-core prefill kernel expired"
-    return out.to(torch.float64).cpu().numpy()
 
 
 def _check(oracle, wl, what="", with_workspace=False):
