@@ -381,6 +381,7 @@ def run_ours(args):
         result["cpu_baseline"] = cpu_baseline(wl, tp_req, tp_idx, outs_d[0].to(torch.float64).cpu().numpy(), budget_s=20.0)
         if not args.no_extras:
             result["extras"] = extras(b, torch, dev, args)
+            result["roofline"]["others"] = roofline_others(result["extras"], peak)
     if world > 1:
         dist.destroy_process_group()
     return result
@@ -711,6 +712,54 @@ def extras(b, torch, dev, args):
     return res
 
 
+def roofline_others(ex, hbm_peak):
+    """The other measured kernels of the path, in the shape of the `roofline` object: one entry per
+    (kernel, workload), taken from the `extras` measurements (L2 flushed before every launch)."""
+    tf_burst, tf_sust = 1609.8, 1365.0
+    try:
+        d = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+        tf_burst, tf_sust = float(d["bf16_tflops"]), float(d["bf16_tflops_sustained"])
+    except Exception:
+        pass
+    out = []
+
+    def hbm(kernel, workload, us, gbps, **kw):
+        out.append({"kernel": kernel, "bound": "hbm", "achieved": gbps, "peak": hbm_peak, "unit": "GB/s",
+                    "frac": round(gbps / hbm_peak, 4), "frac_of_8000_nominal": round(gbps / 8000.0, 4), "us": us,
+                    "workload": workload, **kw})
+    sw = ex.get("decode_sweep", {})
+    names = {"f=0.0:native": "decode_ring_kernel<128,false> (native path)", "f=0.0:elastic_idle": "decode_ring_kernel<128,true> on an all-TARGET pool",
+             "f=0.25:elastic": "decode_ring_kernel<128,true>", "f=0.5:elastic": "decode_ring_kernel<128,true>", "f=1.0:elastic": "decode_ring_kernel<128,true>"}
+    for key, kname in names.items():
+        if key in sw:
+            hbm(kname, f"llama3-8b-shaped decode, batch 64, BASE fraction {key.split(':')[0][2:]}; split kernel alone",
+                sw[key]["split_kernel_us"], sw[key]["split_kernel_GBps"], call_us=sw[key]["us"], call_GBps=sw[key]["GBps"])
+    for key, e in ex.get("other_decode_configs", {}).items():
+        hbm("ekv_attn_decode (split + merge kernels)", key, e["us"], e["GBps"])
+    for key, e in ex.get("batch_ctx_sweep", {}).items():
+        hbm("ekv_attn_decode (split + merge kernels)", f"fixed lengths, f = 0.5: {key}", e["us"], e["GBps"])
+    for key, kname in (("downgrade", "downgrade_pack_kernel + commit"), ("refine", "refine_expand_kernel + commit")):
+        if key in ex:
+            hbm(kname, f"{ex[key]['pairs']} pairs, 1 layer", ex[key]["us"], ex[key]["GBps"])
+        t4 = ex.get("transitions_4_layers", {})
+        if key in t4:
+            hbm(kname, f"{t4['pairs']} pairs, {t4['layers']} layers", t4[key]["us"], t4[key]["GBps"])
+    pl = ex.get("pressure_step_loop", {}).get("steady_state_median")
+    if pl:
+        hbm("downgrade_pack_kernel (last CTA publishes)", f"pressure step loop, {pl['downgrade_pairs']} pairs per step", pl["downgrade_us"], pl["downgrade_GBps"])
+        hbm("ekv_attn_decode (split + merge kernels)", "pressure step loop, batch 256", pl["decode_us"], pl["decode_GBps"])
+        hbm("refine_expand_kernel (last CTA publishes)", f"pressure step loop, {pl['refine_pairs']} pairs per step", pl["refine_us"], pl["refine_GBps"])
+    for key, label in (("prefill_chunk", "bf16"), ("prefill_chunk_fp16", "fp16")):
+        pf = ex.get(key) if key == "prefill_chunk" else ex.get("fp16_elements", {}).get("prefill_chunk")
+        if pf:
+            out.append({"kernel": f"prefill_ws_kernel ({label} elements)", "bound": "tensor", "achieved": pf["TFLOPs"], "peak": tf_burst,
+                        "unit": "TFLOP/s", "frac": round(pf["TFLOPs"] / tf_burst, 4), "peak_sustained": tf_sust,
+                        "frac_of_sustained": round(pf["TFLOPs"] / tf_sust, 4), "us": round(pf["ms"] * 1e3, 1),
+                        "workload": "chunked prefill: batch 8, 512-token chunk over an 8192-token prefix (50 % BASE), 32/8 heads, D 128; "
+                                    "L2 flushed before every launch"})
+    return out
+
+
 def run_prefill_only(args):
     """Chunked prefill against a mixed prefix (configuration 5) alone, for profiling captures."""
     import torch
@@ -778,6 +827,7 @@ def run_decode_only(args):
     kms = float(np.median(ks[1:])) if len(ks) > 1 else ks[0]
     return {"metric": "decode_split_kernel_GBps", "unit": "GB/s", "base_fraction": f, "batch": wl.batch,
             "kv_bytes": int(wl.kv_bytes()), "split_kernel_us": round(kms * 1e3, 1),
+            "split_kernel_us_mean": round(float(np.mean(ks[2:])) * 1e3, 2) if len(ks) > 3 else None,
             "value": round(wl.kv_bytes() / kms / 1e6, 1)}
 
 
@@ -888,7 +938,27 @@ def run_reference(args):
             "gpu_launches": 0}
 
 
-def main():
+def run_plumbing_check(args):
+    """What every rank of a multi-GPU run does around its kernels, with the kernels left out and the
+    gloo backend on CPU: rendezvous from the launcher's environment, rank-specific workload draw,
+    barrier, max over ranks of the (here: made-up, rank-dependent) step time, sum of the bytes."""
+    import torch.distributed as dist
+    world, rank, _ = _dist()
+    if world > 1:
+        dist.init_process_group("gloo")
+    wl = synth.cfg_llama8b_decode(seed=synth.BASE_SEED + 2 + 1000 * rank, base_fraction=0.5, batch=2)
+    step_bytes = float(wl.kv_bytes())
+    if world > 1:
+        dist.barrier()
+    ms, total = aggregate_over_ranks(1.0 + rank, step_bytes)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return {"plumbing_check": True, "n_gpus": world, "ms_per_step": ms, "bytes_all_ranks": total, "bytes_rank0": step_bytes,
+            "scaling": "weak", "backend": "gloo"}
+
+
+def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=2000)
@@ -906,11 +976,26 @@ def main():
                     help="16-bit element type of the pool in the --profile-prefill / --profile-decode modes")
     ap.add_argument("--profile-transitions", action="store_true",
                     help="run only ekv_downgrade / ekv_refine on all eligible pairs of --batch requests (default 32)")
-    args = ap.parse_args()
+    ap.add_argument("--plumbing-check", action="store_true",
+                    help="multi-rank plumbing only, on CPU with the gloo backend: launch, rendezvous, barrier, "
+                         "max-over-ranks time, summed bytes, one JSON line from rank 0; no kernel runs")
+    args = ap.parse_args(argv)
     world, rank, _ = _dist()
-    if args.gpus != world and world == 1 and args.gpus > 1:
-        raise SystemExit("for --gpus N > 1 launch with: python -m torch.distributed.run --nnodes=1 "
-                         "--nproc-per-node N --master-addr 127.0.0.1 --master-port P bench.py --gpus N ...")
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # Launched plainly with --gpus N: start the N ranks (one process per GPU) under torch's launcher
+        # and hand them the same arguments.
+        import socket
+        with socket.socket() as sock:
+            sock.bind(("127.0.0.1", 0))
+            port = sock.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(sys.argv[1:] if argv is None else argv)
+        raise SystemExit(subprocess.call(cmd))
+    if args.plumbing_check:
+        res = run_plumbing_check(args)
+        if rank == 0:
+            print(json.dumps(res), flush=True)
+        return
     if args.profile_prefill:
         res = run_prefill_only(args)
     elif args.profile_transitions:

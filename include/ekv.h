@@ -113,6 +113,16 @@ const char *ekv_status_string(int status);
  *   "prefill_variant"     : 0 (default) = warp-specialised tcgen05 tensor-core kernel at
  *                           head_dim 128, mma.sync kernel otherwise; 1 = always the mma.sync
  *                           kernel (comparator).
+ *   "decode_two_term"     : how the decode kernels treat the 16-bit rounding of the probabilities that
+ *                           enter the PV product: 0 (default) = a step that holds a token with an eighth
+ *                           or more of the probability mass its warp has seen so far takes PV a second
+ *                           time with the rounding residuals; 1 = never (one-term product: the output's
+ *                           error before its final rounding can then reach 5e-3 on rows that two or
+ *                           three tokens dominate); 2 = every step. For measurements.
+ *   "attn_out_f32"        : debug aid, 0 (default) or 1: the attention entry points (decode, its
+ *                           structured and no-workspace forms, prefill) then treat `out` as a float32
+ *                           array of the same shape and store the result as it stands before the
+ *                           rounding to the 16-bit output type.
  * Returns EKV_OK or EKV_ERR_INVALID_ARG for an unknown name / bad value. */
 int ekv_set_option(const char *name, int64_t value);
 
@@ -148,17 +158,53 @@ int ekv_attn_decode(const ekv_pool *pool, int32_t layer, const ekv_batch *batch,
                     const void *q, void *out, int32_t num_q_heads, float sm_scale,
                     int32_t max_seq_len, void *workspace, size_t workspace_bytes, void *stream);
 
-/* Metadata lowering (Sec. 3.2: mixed sequences commonly form a TARGET-BASE-TARGET layout with at
- * most two mode boundaries; App. B.3: the worker inspects the mode layout and lowers it into
- * `elastic_boundaries` for regular sequences). From the per-block tags of a batch, writes for
- * every request the pair-index range that is BASE: boundaries[2r] = first BASE pair,
- * boundaries[2r+1] = one past the last BASE pair (0, 0 when the request has none), and two
- * batch flags: flags[0] = 1 if any request has a BASE pair (the batch-level indicator),
- * flags[1] = 1 if any request is irregular (a TARGET pair between two BASE pairs), in which case
- * the boundaries do not describe that request and the general path must be used.
+/* Mode boundaries from the tags (Sec. 3.2, structured path; App. B.3). A "regular" sequence has
+ * all its BASE pairs in one contiguous run of pair indices, so two integers describe its modes.
+ * From the per-block tags of a batch this call writes, for every request, that run:
+ * boundaries[2r] = first BASE pair, boundaries[2r+1] = one past the last BASE pair (0, 0 when the
+ * request has none), and two batch flags: flags[0] = 1 if any request has a BASE pair (the
+ * batch-level indicator), flags[1] = 1 if any request is irregular (a TARGET pair between two BASE
+ * pairs), in which case the boundaries do not describe that request and the general path must be
+ * used.
  *   boundaries : device int32 [batch][2];  flags : device int32 [2] (cleared by this call) */
 int ekv_lower_metadata(const ekv_pool *pool, const ekv_batch *batch, int32_t *boundaries,
                        int32_t *flags, void *stream);
+
+/* Lowering of the scheduler's sparse per-request metadata (Sec. 3.4; App. B.3: the scheduler emits
+ * sparse BASE metadata per request and the worker lowers it into device tensors). The scheduler
+ * describes scheduled request i by its sequence length, its logical -> physical block list (for a
+ * BASE pair both entries name the block that stores the pair) and a short, sorted list of disjoint
+ * pair-index ranges [first, one past last) that are BASE. One kernel launch writes what the
+ * attention entry points read:
+ *   block_table row row_of[i] : entries [0, n_blocks_i) = the block list (later entries untouched)
+ *   seq_lens_out[row_of[i]]   : lens[i]
+ *   boundaries[row_of[i]]     : first BASE pair, one past the last BASE pair (0, 0 without ranges)
+ *   flags[0] : 1 if any request has a range;  flags[1] : 1 if any request has two ranges with a gap
+ *              between them (irregular: use the general path, not ekv_attn_decode_structured)
+ * and cross-checks the description against the tags, which the transition kernels own:
+ *   flags[2] : number of pairs whose tag disagrees with the ranges (BASE tag outside every range,
+ *              TARGET tag inside one, a BASE pair whose two entries differ, a TARGET pair whose
+ *              entries coincide, a block id out of range)
+ *   flags[3] : 0 if flags[2] == 0, else n_req minus the index i of the first such request
+ * Nothing else is read or written; tags are never modified.
+ *   batch       : block_table and max_blocks are used (seq_lens is not; pass the output separately)
+ *   row_of      : device int32 [n_req] table row of each scheduled request, or NULL for row i = i
+ *   lens        : device int32 [n_req]
+ *   blk_start   : device int32 [n_req+1] offsets into blk_ids;  blk_ids : device int32 [blk_start[n_req]]
+ *   range_start : device int32 [n_req+1] offsets into ranges;   ranges  : device int32 [..][2]
+ *   boundaries  : device int32 [batch][2];  flags : device int32 [4] (cleared by this call)
+ * The inputs can be views of one buffer, so a step's metadata travels in one host-to-device copy. */
+int ekv_lower_sparse_metadata(const ekv_pool *pool, const ekv_batch *batch, int32_t *seq_lens_out,
+                              int32_t n_req, const int32_t *row_of, const int32_t *lens,
+                              const int32_t *blk_start, const int32_t *blk_ids,
+                              const int32_t *range_start, const int32_t *ranges,
+                              int32_t *boundaries, int32_t *flags, void *stream);
+
+/* Tags of released blocks (Sec. 3.1: a released physical block carries no fidelity): sets
+ * tags[block_ids[i]] = EKV_TARGET for i < n, e.g. for the blocks of a finished request that stored
+ * BASE pairs, before the allocator hands them out again.
+ *   block_ids : device int32 [n] */
+int ekv_reset_tags(const ekv_pool *pool, const int32_t *block_ids, int32_t n, void *stream);
 
 /* Structured elastic decode path (Sec. 3.2; App. B.3): same computation and arguments as
  * ekv_attn_decode for a batch with has_base != 0 whose sequences all have the regular
@@ -215,8 +261,8 @@ int ekv_attn_prefill_chunk(const ekv_pool *pool, int32_t layer, const ekv_batch 
                            int32_t total_q, int32_t max_q_len, int32_t max_seq_len,
                            void *workspace, size_t workspace_bytes, void *stream);
 
-/* KV append (Sec. 3.2 / App. B.3: newly appended KV is written in TARGET form and stays in the
- * protected recent region until it becomes eligible for demotion). Request r contributes
+/* KV append (Sec. 3.2 / App. B.3): new tokens always enter the pool as full 16-bit words, in
+ * TARGET blocks; demotion only ever touches older pairs. Request r contributes
  * C_r = q_start[r+1] - q_start[r] new tokens, the last C_r of its seq_lens[r] tokens; token i of
  * the chunk is written at position seq_lens[r] - C_r + i, i.e. into slot position % 16 of the
  * physical block that block_table maps logical block position / 16 to (TARGET layout). One

@@ -78,9 +78,11 @@ int ekv_ctrl_plan_demotion(ekv_ctrl *c, int32_t demand, int32_t *pair_req, int32
  * released blocks join the free list, E_t is recorded. */
 int ekv_ctrl_commit_demotion(ekv_ctrl *c, int32_t n, const int32_t *freed_blocks);
 
-/* Step t, after required scheduling and allocation: advances the reserve (R_t), computes the
- * promotion budget P_t from the current free count and picks min(P_t, transfer_slack) BASE
- * pairs. Each reserves one free block now (new_blocks[i]). In flight until commit. */
+/* Step t, after required scheduling and allocation: advances the reserve (R_t; once per step,
+ * however often this is called; a step in which it is not called at all has its update applied
+ * when the next ekv_ctrl_plan_demotion opens the following step), computes the promotion budget
+ * P_t from the current free count and picks min(P_t, transfer_slack) BASE pairs. Each reserves
+ * one free block now (new_blocks[i]). In flight until commit. */
 int ekv_ctrl_plan_promotion(ekv_ctrl *c, int32_t transfer_slack, int32_t *pair_req, int32_t *pair_idx,
                             int32_t *new_blocks, int32_t *resid_slot, int32_t cap, int32_t *n_out);
 /* After ekv_refine completed (or was enqueued on the stream all consumers use): the first n

@@ -1,7 +1,10 @@
-"""TEST INFRASTRUCTURE. The scalar recurrences of the paper's Algorithm 1 ("Pressure-aware fidelity
-control", Sec. 3.3), written out step by step in the paper's notation, for checking the host
-controller. Only counts, no block ids: which pairs are picked is a ranking choice the paper
-leaves to the runtime; how many, and the reserve and budget that follow, are fixed by it."""
+"""TEST INFRASTRUCTURE. The five scalar quantities that Algorithm 1 (Sec. 3.3) fixes for one
+scheduling step (shortage, demotion count, surplus, reserve, promotion budget), as one function
+over counts, for checking the host controller on random traces. Which pairs are picked is a
+ranking choice the paper leaves to the runtime; only how many is fixed. The function is pinned by
+hand-computed steps and by the properties the section states (tests/test_controller.py: bounds of
+the demotion count, reserve at least the surplus, decay to zero in ceil(R / lambda) idle steps,
+budget = free blocks beyond the reserve)."""
 
 
 def step(D_t, F_t, eligible_target_pairs, R_prev, B_min_d, lam, blocks_allocated, eligible_base_pairs,

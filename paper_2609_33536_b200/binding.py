@@ -17,7 +17,7 @@ EXPORTS = ("ekv_version", "ekv_status_string", "ekv_set_option", "ekv_set_profil
            "ekv_attn_decode", "ekv_attn_prefill_chunk", "ekv_downgrade", "ekv_refine",
            "ekv_validate_batch", "ekv_attn_decode_noalloc", "ekv_attn_decode_noalloc_max_bytes",
            "ekv_prefill_status", "ekv_lower_metadata", "ekv_attn_decode_structured",
-           "ekv_kv_append")
+           "ekv_kv_append", "ekv_lower_sparse_metadata", "ekv_reset_tags")
 
 
 class EkvError(RuntimeError):
@@ -80,6 +80,10 @@ def load(path: str | None = None):
         L.ekv_attn_decode_structured.argtypes = [PP, i32, BP, vp, vp, vp, i32, f32, i32, vp, sz, vp]
         L.ekv_kv_append.restype = C.c_int
         L.ekv_kv_append.argtypes = [PP, i32, BP, vp, vp, vp, i32, vp, vp]
+        L.ekv_lower_sparse_metadata.restype = C.c_int
+        L.ekv_lower_sparse_metadata.argtypes = [PP, BP, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.ekv_reset_tags.restype = C.c_int
+        L.ekv_reset_tags.argtypes = [PP, vp, i32, vp]
         L.ekv_prefill_status.restype = C.c_int
         L.ekv_validate_batch.restype = C.c_int
         L.ekv_validate_batch.argtypes = [PP, BP, vp, vp]
@@ -180,6 +184,22 @@ def ekv_lower_metadata(pool: Pool, batch: Batch, boundaries, flags):
     """boundaries: int32 [batch][2] out; flags: int32 [2] out (has_base, any_irregular)."""
     _check(load().ekv_lower_metadata(C.byref(pool.c), C.byref(batch.c), _ptr(boundaries), _ptr(flags), _stream()),
            "ekv_lower_metadata")
+
+
+def ekv_lower_sparse_metadata(pool: Pool, batch: Batch, seq_lens_out, row_of, lens, blk_start, blk_ids,
+                              range_start, ranges, boundaries, flags):
+    """Scheduler-side sparse description (block lists + BASE pair ranges, CSR) -> block-table rows,
+    sequence lengths, boundaries [batch][2], flags [4] (any BASE, any irregular, disagreeing pairs,
+    n_req - first disagreeing request)."""
+    _check(load().ekv_lower_sparse_metadata(C.byref(pool.c), C.byref(batch.c), _ptr(seq_lens_out), int(lens.numel()),
+                                            _ptr(row_of), _ptr(lens), _ptr(blk_start), _ptr(blk_ids), _ptr(range_start),
+                                            _ptr(ranges), _ptr(boundaries), _ptr(flags), _stream()),
+           "ekv_lower_sparse_metadata")
+
+
+def ekv_reset_tags(pool: Pool, block_ids):
+    """tags[block_ids] = TARGET for blocks that leave their request."""
+    _check(load().ekv_reset_tags(C.byref(pool.c), _ptr(block_ids), int(block_ids.numel()), _stream()), "ekv_reset_tags")
 
 
 def ekv_attn_decode_structured(pool: Pool, layer: int, batch: Batch, boundaries, q, out, num_q_heads: int,

@@ -2,6 +2,7 @@
 // the device-side batch checker.
 #include "ekv_common.cuh"
 #include <string.h>
+#include <atomic>
 
 namespace ekv {
 
@@ -10,7 +11,22 @@ int64_t g_decode_variant = 0;
 int64_t g_decode_merge_slices = 0;
 int64_t g_prefill_variant = 0;
 int64_t g_attn_out_f32 = 0;
+int64_t g_decode_two_term = 0;
 void *g_profile_ev[2] = {nullptr, nullptr};
+
+int device_sm_count()
+{
+    constexpr int kMaxDevices = 64;
+    static std::atomic<int> cache[kMaxDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return kSmCountB200;
+    int v = cache[dev].load(std::memory_order_relaxed);
+    if (v == 0) {
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return kSmCountB200;
+        cache[dev].store(v, std::memory_order_relaxed);
+    }
+    return v;
+}
 
 __global__ void validate_batch_kernel(const int32_t *block_table, const int32_t *seq_lens, const uint8_t *tags,
                                       int batch, int max_blocks, int num_blocks, int has_base, int32_t *status)
@@ -76,6 +92,11 @@ extern "C" int ekv_set_option(const char *name, int64_t value)
     if (!strcmp(name, "attn_out_f32")) {
         if (value != 0 && value != 1) return EKV_ERR_INVALID_ARG;
         g_attn_out_f32 = value;
+        return EKV_OK;
+    }
+    if (!strcmp(name, "decode_two_term")) {
+        if (value < 0 || value > 2) return EKV_ERR_INVALID_ARG;
+        g_decode_two_term = value;
         return EKV_OK;
     }
     if (!strcmp(name, "decode_variant")) {

@@ -9,13 +9,15 @@
 namespace ekv {
 
 constexpr int kPageSize = 16;
-constexpr int kSmCount = 148;
+constexpr int kSmCountB200 = 148;        // fallback when the device cannot be queried
+int device_sm_count();                   // SMs of the current device (cached per device)
 
 extern int64_t g_decode_chunk_tokens;   // option "decode_chunk_tokens"; 0 = automatic
 extern int64_t g_prefill_variant;       // option "prefill_variant"; 0 = automatic (tcgen05 kernel at head_dim 128), 1 = mma.sync kernel
 extern void *g_profile_ev[2];           // ekv_set_profile_events: recorded around the main kernel of a call
 extern int64_t g_decode_merge_slices;   // option "decode_merge_slices"; 0 = automatic, else 1, 4 or 8
 extern int64_t g_attn_out_f32;          // option "attn_out_f32"; 1 = attention entry points store fp32 outputs (debug)
+extern int64_t g_decode_two_term;       // option "decode_two_term"; 0 = by the mass test (default), 1 = never, 2 = every step
 extern int64_t g_decode_variant;        // option "decode_variant"; 0 / 3 = ring-staged kernel, 1 = page-stepped comparator
 int decode_chunk_tokens(int batch, int num_kv_heads, int max_seq_len);
 size_t decode_workspace_bytes(int batch, int num_q_heads, int num_kv_heads, int head_dim, int max_seq_len);

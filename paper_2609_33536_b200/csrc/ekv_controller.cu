@@ -35,6 +35,7 @@ struct ekv_ctrl {
     std::vector<int> free_slots;
     std::vector<Item> demoting, promoting;
     int64_t step = 0;
+    int64_t reserve_step = -1;   // step whose reserve update (R_t) has been applied
     int reserve = 0, shortage = 0, surplus = 0, pending_surplus = 0, budget = 0, base_pairs = 0;
 
     int blocks_for(int n_tokens) const { return (n_tokens + cfg.page_size - 1) / cfg.page_size; }
@@ -136,14 +137,24 @@ extern "C" int32_t ekv_ctrl_demand_for(const ekv_ctrl *c, int32_t req, int32_t n
     return std::max(0, c->blocks_for(new_n_tokens) - have);
 }
 
+// R_t = max(0, R_{t-1} - lambda) + E_t, applied exactly once per step: by the step's promotion plan,
+// or, when a step has none, when the next step begins.
+static void advance_reserve(ekv_ctrl *c)
+{
+    if (c->reserve_step == c->step) return;
+    c->reserve = std::max(0, c->reserve - c->cfg.reserve_decay) + c->pending_surplus;
+    c->pending_surplus = 0;
+    c->reserve_step = c->step;
+}
+
 extern "C" int ekv_ctrl_plan_demotion(ekv_ctrl *c, int32_t demand, int32_t *pair_req, int32_t *pair_idx,
                                       int32_t *resid_slot, int32_t cap, int32_t *n_out)
 {
     if (!c || !n_out || demand < 0) return EKV_CTRL_ERR_ARG;
     if (!c->demoting.empty()) return EKV_CTRL_ERR_STATE;
+    advance_reserve(c);             // a step that ended without a promotion plan still ages the reserve once
     ++c->step;
     *n_out = 0;
-    c->pending_surplus = 0;
     const int free_now = (int)c->free_blocks.size();
     c->shortage = std::max(0, demand - free_now);                       // Delta_t
     if (c->shortage == 0) return EKV_CTRL_OK;
@@ -204,8 +215,7 @@ extern "C" int ekv_ctrl_plan_promotion(ekv_ctrl *c, int32_t transfer_slack, int3
     if (!c->demoting.empty()) return EKV_CTRL_ERR_STATE;               // demotion of this step not committed yet
     *n_out = 0;
     // R_t = max(0, R_{t-1} - lambda) + E_t ;  P_t = max(0, F_post - R_t)
-    c->reserve = std::max(0, c->reserve - c->cfg.reserve_decay) + c->pending_surplus;
-    c->pending_surplus = 0;
+    advance_reserve(c);
     c->budget = std::max(0, (int)c->free_blocks.size() - c->reserve);
     int n_p = std::min(c->budget, transfer_slack);
     if (n_p == 0) return EKV_CTRL_OK;

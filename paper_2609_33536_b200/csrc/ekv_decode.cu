@@ -48,9 +48,13 @@ struct DecodeParams {
     int chunk_tokens, max_splits;
     float scale_log2;                   // sm_scale * log2(e)
     int out_f32;                        // debug: `out` is float [batch][Hq][D] and receives the unrounded result
+    int two_term;                       // 0 = two-term probabilities by the mass test, 1 = never, 2 = on every step
 };
 
 __device__ __forceinline__ bool m_run_is_empty(float m) { return m == -INFINITY; }
+
+constexpr int kTwoTermRefresh = 8;             // steps between refreshes of the two-term threshold (see softmax_step_t)
+constexpr float kTwoTermLog2Share = -3.0f;     // log2 of the probability share from which a token gets a two-term probability
 
 template <int BYTES> struct Loader;
 template <> struct Loader<64> { template <int N> static __device__ __forceinline__ void ld(const uint8_t *p, uint32_t (&r)[N], int at) {
@@ -121,6 +125,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 3) decode_page_kernel(DecodePa
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) { o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f; }
     float m_run = -INFINITY, l_run = 0.f;
+    float thr_abs = p.two_term == 1 ? INFINITY : -INFINITY;   // two-term threshold of head c (absolute score units)
 
     const int32_t *bt_row = p.block_table + (int64_t)r * p.max_blocks;
     int packed = 0;                                    // lane i: (phys << 1 | tag) of iteration base+i
@@ -229,6 +234,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 3) decode_page_kernel(DecodePa
         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
         const float m_new = fmaxf(m_run, mx);                   // finite: token 0 of a page is valid
+        const bool two_term = __any_sync(0xffffffffu, !(mx < thr_abs));   // see softmax_step_t: p = hi + lo for steps with a heavy token
         const float alpha = fast_exp2(m_run - m_new);
         float pr[2][2];
 #pragma unroll
@@ -240,6 +246,14 @@ __global__ void __launch_bounds__(kDecodeThreads, 3) decode_page_kernel(DecodePa
         m_run = m_new;
         const uint32_t pb0 = pack_bf16x2(pr[0][0], pr[0][1]);
         const uint32_t pb1 = pack_bf16x2(pr[1][0], pr[1][1]);
+        uint32_t pl0 = 0u, pl1 = 0u;
+        if (two_term) {
+            float h0, h1;
+            unpack_16x2<false>(pb0, h0, h1);
+            pl0 = pack_bf16x2(pr[0][0] - h0, pr[0][1] - h1);
+            unpack_16x2<false>(pb1, h0, h1);
+            pl1 = pack_bf16x2(pr[1][0] - h0, pr[1][1] - h1);
+        }
         // rescale factors of the two heads this lane holds in O^T (columns 2j, 2j+1)
         const float al0 = __shfl_sync(0xffffffffu, alpha, (2 * j) * 4);
         const float al1 = __shfl_sync(0xffffffffu, alpha, (2 * j + 1) * 4);
@@ -276,24 +290,39 @@ __global__ void __launch_bounds__(kDecodeThreads, 3) decode_page_kernel(DecodePa
                 // [t0.b1, t0.b0, t1.b1, t1.b0] and the same for bytes 3,2
                 const uint32_t ul = prmt(x0, x1, 0x4501), uh = prmt(x0, x1, 0x6723);
                 const uint32_t wl = prmt(x2, x3, 0x4501), wh = prmt(x2, x3, 0x6723);
-                mma_16816(o[2 * qd][0], o[2 * qd][1], o[2 * qd][2], o[2 * qd][3],
-                          ul & 0xFF00FF00u, prmt(ul, 0u, 0x2404), wl & 0xFF00FF00u, prmt(wl, 0u, 0x2404),
+                const uint32_t a0 = ul & 0xFF00FF00u, a1 = prmt(ul, 0u, 0x2404), a2 = wl & 0xFF00FF00u, a3 = prmt(wl, 0u, 0x2404);
+                const uint32_t b0 = uh & 0xFF00FF00u, b1 = prmt(uh, 0u, 0x2404), b2 = wh & 0xFF00FF00u, b3 = prmt(wh, 0u, 0x2404);
+                mma_16816(o[2 * qd][0], o[2 * qd][1], o[2 * qd][2], o[2 * qd][3], a0, a1, a2, a3,
                           pb0, pb1, o[2 * qd][0], o[2 * qd][1], o[2 * qd][2], o[2 * qd][3]);
-                mma_16816(o[2 * qd + 1][0], o[2 * qd + 1][1], o[2 * qd + 1][2], o[2 * qd + 1][3],
-                          uh & 0xFF00FF00u, prmt(uh, 0u, 0x2404), wh & 0xFF00FF00u, prmt(wh, 0u, 0x2404),
+                mma_16816(o[2 * qd + 1][0], o[2 * qd + 1][1], o[2 * qd + 1][2], o[2 * qd + 1][3], b0, b1, b2, b3,
                           pb0, pb1, o[2 * qd + 1][0], o[2 * qd + 1][1], o[2 * qd + 1][2], o[2 * qd + 1][3]);
+                if (two_term) {
+                    mma_16816(o[2 * qd][0], o[2 * qd][1], o[2 * qd][2], o[2 * qd][3], a0, a1, a2, a3,
+                              pl0, pl1, o[2 * qd][0], o[2 * qd][1], o[2 * qd][2], o[2 * qd][3]);
+                    mma_16816(o[2 * qd + 1][0], o[2 * qd + 1][1], o[2 * qd + 1][2], o[2 * qd + 1][3], b0, b1, b2, b3,
+                              pl0, pl1, o[2 * qd + 1][0], o[2 * qd + 1][1], o[2 * qd + 1][2], o[2 * qd + 1][3]);
+                }
             }
         } else {
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) {
                 const uint32_t x0 = vr[0 * VREG_T + mt], x1 = vr[1 * VREG_T + mt];
                 const uint32_t x2 = vr[2 * VREG_T + mt], x3 = vr[3 * VREG_T + mt];
-                mma_16816(o[mt][0], o[mt][1], o[mt][2], o[mt][3],
-                          prmt(x0, x1, 0x5410), prmt(x0, x1, 0x7632), prmt(x2, x3, 0x5410), prmt(x2, x3, 0x7632),
+                const uint32_t a0 = prmt(x0, x1, 0x5410), a1 = prmt(x0, x1, 0x7632), a2 = prmt(x2, x3, 0x5410), a3 = prmt(x2, x3, 0x7632);
+                mma_16816(o[mt][0], o[mt][1], o[mt][2], o[mt][3], a0, a1, a2, a3,
                           pb0, pb1, o[mt][0], o[mt][1], o[mt][2], o[mt][3]);
+                if (two_term)
+                    mma_16816(o[mt][0], o[mt][1], o[mt][2], o[mt][3], a0, a1, a2, a3,
+                              pl0, pl1, o[mt][0], o[mt][1], o[mt][2], o[mt][3]);
             }
         }
         cur = nxt;
+        if (p.two_term == 0 && ((it & (it + 1)) == 0 || (it & (kTwoTermRefresh - 1)) == kTwoTermRefresh - 1)) {
+            float L = l_run;
+            L += __shfl_xor_sync(0xffffffffu, L, 1);
+            L += __shfl_xor_sync(0xffffffffu, L, 2);
+            thr_abs = m_run + __log2f(L) + kTwoTermLog2Share;
+        }
     }
 
     // ---- merge the warps of this CTA ----
@@ -400,9 +429,23 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a)
     asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
     return d;
 }
+// Two-term probabilities. P enters the PV product as a 16-bit float; on a row that a few tokens
+// dominate the rounding of those few probabilities (2^-9 relative for bf16) is what remains of the
+// output error, up to 5e-3 absolute. When a step holds a token that can end up with an eighth or
+// more of a head's probability mass, its probabilities are therefore split as p = hi + lo (both
+// 16-bit, lo = the rounding residual, exact in fp32) and PV is taken for both terms. The test must
+// not miss such a token, and is cheap: a token's final share is at most p / L, L being any lower
+// bound of the head's final probability mass, so "step maximum >= thr_abs" with
+// thr_abs = log2(L / 8) in absolute score units (which do not move with the running maximum) is a
+// necessary condition. L is the mass this warp has seen so far (a warp's own sums only: the decision
+// must not depend on how far other warps have got, or results would differ from run to run),
+// refreshed after steps 0, 1, 3, 7 and then every kTwoTermRefresh steps; between refreshes the
+// mass only grows, which makes the stale threshold the stricter one. Before the first refresh
+// every step takes two terms.
 template <int MTILES, bool QUAD_TOKENS, bool F16>
 __device__ __forceinline__ void softmax_step_t(float (&s)[MTILES][4], int valid, int g, float (&m_run)[2], float (&l_run)[2],
-                                               uint32_t (&pb)[2 * MTILES], float (&alpha)[2])
+                                               uint32_t (&pb)[2 * MTILES], float (&alpha)[2],
+                                               const float (&thr_abs)[2], bool &two_term, uint32_t save_addr)
 {
     if (valid < MTILES * 16) {
 #pragma unroll
@@ -413,6 +456,10 @@ __device__ __forceinline__ void softmax_step_t(float (&s)[MTILES][4], int valid,
                 if (tok >= valid) s[mt][2 * half] = s[mt][2 * half + 1] = -INFINITY;
             }
     }
+    // the masked scores are parked in this lane's shared-memory slot: the rare two-term pass takes them from there
+#pragma unroll
+    for (int mt = 0; mt < MTILES; ++mt)
+        asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" :: "r"(save_addr + 16 * mt), "f"(s[mt][0]), "f"(s[mt][1]), "f"(s[mt][2]), "f"(s[mt][3]) : "memory");
     float mx[2];
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
@@ -425,6 +472,7 @@ __device__ __forceinline__ void softmax_step_t(float (&s)[MTILES][4], int valid,
         mx[0] = fmaxf(mx[0], __shfl_xor_sync(0xffffffffu, mx[0], o));
         mx[1] = fmaxf(mx[1], __shfl_xor_sync(0xffffffffu, mx[1], o));
     }
+    two_term = __any_sync(0xffffffffu, !(mx[0] < thr_abs[0]) || !(mx[1] < thr_abs[1]));
     float sum[2] = {0.f, 0.f};
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
@@ -443,6 +491,25 @@ __device__ __forceinline__ void softmax_step_t(float (&s)[MTILES][4], int valid,
     }
     l_run[0] = l_run[0] * alpha[0] + sum[0];
     l_run[1] = l_run[1] * alpha[1] + sum[1];
+}
+
+// The low-order terms of a step's probabilities, recomputed from the parked scores with the running
+// maxima the step ended on (the same instructions on the same values as in softmax_step_t, so hi is
+// bit for bit what the first pass multiplied with): lo = p - hi, in B-fragment order like pb.
+template <int MTILES, bool F16>
+__device__ __forceinline__ void two_term_residuals(uint32_t save_addr, const float (&m_run)[2], uint32_t (&pl)[2 * MTILES])
+{
+#pragma unroll
+    for (int mt = 0; mt < MTILES; ++mt) {
+        float s0, s1, s2, s3, h0, h1, h2, h3;
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(s0), "=f"(s1), "=f"(s2), "=f"(s3) : "r"(save_addr + 16 * mt) : "memory");
+        const float p0 = fast_exp2(s0 - m_run[0]), p1 = fast_exp2(s1 - m_run[1]);
+        const float p2 = fast_exp2(s2 - m_run[0]), p3 = fast_exp2(s3 - m_run[1]);
+        unpack_16x2<F16>(pack_16x2<F16>(p0, p1), h0, h1);
+        unpack_16x2<F16>(pack_16x2<F16>(p2, p3), h2, h3);
+        pl[2 * mt] = movmatrix_trans(pack_16x2<F16>(p0 - h0, p1 - h1));
+        pl[2 * mt + 1] = movmatrix_trans(pack_16x2<F16>(p2 - h2, p3 - h3));
+    }
 }
 
 // One step of a warp: a run of tokens that is contiguous in one (block, kv head) slab.
@@ -512,6 +579,7 @@ __global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(D
     float (*sm_m)[8] = (float (*)[8])((uint8_t *)sm_q + KS * 32 * sizeof(uint2));
     float (*sm_l)[8] = sm_m + kDecodeWarps;
     uint2 *sm_steps = (uint2 *)(sm_l + kDecodeWarps);     // [4 warps][64] step descriptors
+    const uint32_t save_addr = (uint32_t)__cvta_generic_to_shared(sm_steps + kDecodeWarps * 64) + threadIdx.x * 32;   // this lane's parked scores of a step
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int c = lane >> 2, j = lane & 3;
@@ -553,6 +621,8 @@ __global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(D
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) { o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f; }
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};     // heads 2j, 2j + 1; sums over this lane's token rows
+    float thr_abs[2] = {-INFINITY, -INFINITY};       // two-term threshold of the two heads (absolute score units); -inf = always
+    if (p.two_term == 1) thr_abs[0] = thr_abs[1] = INFINITY;
 
     // Step list of this warp, built once: a TARGET pair is two steps (one per member that exists), a
     // BASE pair one. Lane i looks at the warp's i-th pair (w, w+4, ...): table entries, tag (or
@@ -700,39 +770,48 @@ __global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(D
             commit();
             uint32_t pb[4];
             float alpha[2];
-            softmax_step_t<2, true, F16>(s, valid, c, m_run, l_run, pb, alpha);
+            bool two_term;
+            softmax_step_t<2, true, F16>(s, valid, c, m_run, l_run, pb, alpha, thr_abs, two_term, save_addr);
             asm volatile("cp.async.wait_group %0;" :: "n"(2 * STAGES - 1) : "memory");  // V of this step landed
             __syncwarp();
             if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) rescale(alpha);      // the running maxima rarely move
             // V: 16 tokens x 16 dims per 8-bit transposing ldmatrix: r0 = tokens 4j..4j+3 of dim c,
             // r1 = the same tokens of dim c + 8; two matrices (two m-tiles) per instruction
+            auto pv_base = [&](const uint32_t (&pf)[4]) {
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                // 0 * NaN must not leak from rows past the end: a token byte past the end is replaced by
-                // the zero byte of the permute's second operand (selector nibble 4)
-                uint32_t sel_lo = 0x1404u, sel_hi = 0x3424u;   // bytes (0, 1) / (2, 3) become high halves
-                if (valid < 32) {
-                    const int rem = valid - (16 * hf + 4 * j);
-                    if (rem < 1) sel_lo = (sel_lo & 0xff0fu) | 0x0040u;      // token 4j
-                    if (rem < 2) sel_lo = (sel_lo & 0x0fffu) | 0x4000u;      // token 4j + 1
-                    if (rem < 3) sel_hi = (sel_hi & 0xff0fu) | 0x0040u;      // token 4j + 2
-                    if (rem < 4) sel_hi = (sel_hi & 0x0fffu) | 0x4000u;      // token 4j + 3
-                }
-                const int vrow = 16 * hf + (lane & 15);
-                const uint32_t rowp = vslot + vrow * (CPR_B * 16);
+                for (int hf = 0; hf < 2; ++hf) {
+                    // 0 * NaN must not leak from rows past the end: a token byte past the end is replaced by
+                    // the zero byte of the permute's second operand (selector nibble 4)
+                    uint32_t sel_lo = 0x1404u, sel_hi = 0x3424u;   // bytes (0, 1) / (2, 3) become high halves
+                    if (valid < 32) {
+                        const int rem = valid - (16 * hf + 4 * j);
+                        if (rem < 1) sel_lo = (sel_lo & 0xff0fu) | 0x0040u;      // token 4j
+                        if (rem < 2) sel_lo = (sel_lo & 0x0fffu) | 0x4000u;      // token 4j + 1
+                        if (rem < 3) sel_hi = (sel_hi & 0xff0fu) | 0x0040u;      // token 4j + 2
+                        if (rem < 4) sel_hi = (sel_hi & 0x0fffu) | 0x4000u;      // token 4j + 3
+                    }
+                    const int vrow = 16 * hf + (lane & 15);
+                    const uint32_t rowp = vslot + vrow * (CPR_B * 16);
 #pragma unroll
-                for (int mp = 0; mp < MT / 2; ++mp) {
-                    const int ch = 2 * mp + (lane >> 4);
-                    uint32_t r0, r1, r2, r3;
-                    ldsm_b8_x2_trans(rowp + (((ch ^ (vrow & 7)) & (CPR_B - 1)) << 4), r0, r1, r2, r3);
-                    mma_16816<F16>(o[2 * mp][0], o[2 * mp][1], o[2 * mp][2], o[2 * mp][3],
-                              prmt(r0, 0u, sel_lo), prmt(r1, 0u, sel_lo), prmt(r0, 0u, sel_hi), prmt(r1, 0u, sel_hi),
-                              pb[2 * hf], pb[2 * hf + 1], o[2 * mp][0], o[2 * mp][1], o[2 * mp][2], o[2 * mp][3]);
-                    mma_16816<F16>(o[2 * mp + 1][0], o[2 * mp + 1][1], o[2 * mp + 1][2], o[2 * mp + 1][3],
-                              prmt(r2, 0u, sel_lo), prmt(r3, 0u, sel_lo), prmt(r2, 0u, sel_hi), prmt(r3, 0u, sel_hi),
-                              pb[2 * hf], pb[2 * hf + 1],
-                              o[2 * mp + 1][0], o[2 * mp + 1][1], o[2 * mp + 1][2], o[2 * mp + 1][3]);
+                    for (int mp = 0; mp < MT / 2; ++mp) {
+                        const int ch = 2 * mp + (lane >> 4);
+                        uint32_t r0, r1, r2, r3;
+                        ldsm_b8_x2_trans(rowp + (((ch ^ (vrow & 7)) & (CPR_B - 1)) << 4), r0, r1, r2, r3);
+                        mma_16816<F16>(o[2 * mp][0], o[2 * mp][1], o[2 * mp][2], o[2 * mp][3],
+                                  prmt(r0, 0u, sel_lo), prmt(r1, 0u, sel_lo), prmt(r0, 0u, sel_hi), prmt(r1, 0u, sel_hi),
+                                  pf[2 * hf], pf[2 * hf + 1], o[2 * mp][0], o[2 * mp][1], o[2 * mp][2], o[2 * mp][3]);
+                        mma_16816<F16>(o[2 * mp + 1][0], o[2 * mp + 1][1], o[2 * mp + 1][2], o[2 * mp + 1][3],
+                                  prmt(r2, 0u, sel_lo), prmt(r3, 0u, sel_lo), prmt(r2, 0u, sel_hi), prmt(r3, 0u, sel_hi),
+                                  pf[2 * hf], pf[2 * hf + 1],
+                                  o[2 * mp + 1][0], o[2 * mp + 1][1], o[2 * mp + 1][2], o[2 * mp + 1][3]);
+                    }
                 }
+            };
+            pv_base(pb);
+            if (two_term) {                                    // rare, uniform over the warp: the low-order terms of P
+                uint32_t pl[4];
+                two_term_residuals<2, F16>(save_addr, m_run, pl);
+                pv_base(pl);
             }
         } else {
             float s[1][4];
@@ -763,12 +842,13 @@ __global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(D
             commit();
             uint32_t pb[2];
             float alpha[2];
-            softmax_step_t<1, false, F16>(s, valid, c, m_run, l_run, pb, alpha);
+            bool two_term;
+            softmax_step_t<1, false, F16>(s, valid, c, m_run, l_run, pb, alpha, thr_abs, two_term, save_addr);
             asm volatile("cp.async.wait_group %0;" :: "n"(2 * STAGES - 1) : "memory");
             __syncwarp();
             if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) rescale(alpha);
             // V: ldmatrix.x4.trans delivers the V^T A-fragments of one m-tile (16 dims x 16 tokens)
-            {
+            auto pv_target = [&](const uint32_t (&pf)[2]) {
                 uint32_t mlo = 0xffffffffu, mhi = 0xffffffffu;     // tokens 2j, 2j+1 | 2j+8, 2j+9
                 if (valid < kPageSize) {
                     mlo = (2 * j < valid ? 0x0000ffffu : 0u) | (2 * j + 1 < valid ? 0xffff0000u : 0u);
@@ -782,14 +862,31 @@ __global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(D
                     uint32_t a0, a1, a2, a3;
                     ldsm_x4_trans(rowp + (((ch ^ (vrow & 7)) & (CPR_T - 1)) << 4), a0, a1, a2, a3);
                     mma_16816<F16>(o[mt][0], o[mt][1], o[mt][2], o[mt][3], a0 & mlo, a1 & mlo, a2 & mhi, a3 & mhi,
-                              pb[0], pb[1], o[mt][0], o[mt][1], o[mt][2], o[mt][3]);
+                              pf[0], pf[1], o[mt][0], o[mt][1], o[mt][2], o[mt][3]);
                 }
+            };
+            pv_target(pb);
+            if (two_term) {
+                uint32_t pl[2];
+                two_term_residuals<1, F16>(save_addr, m_run, pl);
+                pv_target(pl);
             }
         }
         __syncwarp();                                          // every lane is done with this slot
         if (more) issue(nxt, slot, 1);                        // the V slab of this slot is free now
         commit();
         slot = slot + 1 == STAGES ? 0 : slot + 1;
+        if (p.two_term == 0 && ((k & (k + 1)) == 0 || (k & (kTwoTermRefresh - 1)) == kTwoTermRefresh - 1)) {
+            // refresh the two-term thresholds (after steps 0, 1, 3, 7, then every 8th) from the warp-wide sums
+            float L0 = l_run[0], L1 = l_run[1];
+#pragma unroll
+            for (int o = 4; o < 32; o <<= 1) {
+                L0 += __shfl_xor_sync(0xffffffffu, L0, o);
+                L1 += __shfl_xor_sync(0xffffffffu, L1, o);
+            }
+            thr_abs[0] = m_run[0] + __log2f(L0) + kTwoTermLog2Share;
+            thr_abs[1] = m_run[1] + __log2f(L1) + kTwoTermLog2Share;
+        }
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
 
@@ -852,7 +949,7 @@ template <int D, int STAGES>
 constexpr size_t ring_smem_bytes()
 {
     return (size_t)kDecodeWarps * STAGES * (2 * kPageSize * D * 2) + (D / 16) * 32 * sizeof(uint2)
-           + 2 * kDecodeWarps * 8 * sizeof(float) + kDecodeWarps * 64 * sizeof(uint2);
+           + 2 * kDecodeWarps * 8 * sizeof(float) + kDecodeWarps * 64 * sizeof(uint2) + kDecodeThreads * 32;
 }
 
 // Combine the per-split partials of one (request, query head) row: weights 2^(lse_s - max).
@@ -938,7 +1035,7 @@ static cudaError_t launch_merge(const DecodeParams &p, int rows, cudaStream_t st
     // Slices of threads that share a row's splits: as many (8, 4 or 1) as keep the whole grid within
     // one wave of resident threads, and 1 when no row can have more than 8 splits;
     // "decode_merge_slices" overrides.
-    const int64_t wave_threads = (int64_t)kSmCount * 2048;
+    const int64_t wave_threads = (int64_t)device_sm_count() * 2048;
     int sg = (int64_t)rows * D * 8 <= wave_threads ? 8 : ((int64_t)rows * D * 4 <= wave_threads ? 4 : 1);
     if (g_decode_merge_slices > 0) sg = (int)g_decode_merge_slices;
     if (p.max_splits <= 8) sg = 1;
@@ -963,7 +1060,7 @@ int decode_chunk_tokens(int batch, int num_kv_heads, int max_seq_len)
 {
     int64_t chunk = g_decode_chunk_tokens;
     if (chunk <= 0) {
-        const int64_t want_ctas = (int64_t)kSmCount * 3 * 6;
+        const int64_t want_ctas = (int64_t)device_sm_count() * 3 * 6;
         chunk = ((int64_t)max_seq_len * batch * num_kv_heads + want_ctas - 1) / want_ctas;
         if (chunk < 256) chunk = 256;
         if (chunk > kMaxChunkTokens) chunk = kMaxChunkTokens;
@@ -1022,6 +1119,7 @@ static int decode_impl(const ekv_pool *pool, int32_t layer, const ekv_batch *bat
     p.max_splits = max_seq_len > 0 ? (max_seq_len + p.chunk_tokens - 1) / p.chunk_tokens : 1;
     p.scale_log2 = sm_scale * 1.4426950408889634f;
     p.out_f32 = g_attn_out_f32 ? 1 : 0;
+    p.two_term = (int)g_decode_two_term;
     if (p.max_splits > 1) {
         const size_t need = decode_workspace_bytes(batch->batch, num_q_heads, pool->num_kv_heads, pool->head_dim, max_seq_len);
         if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) return EKV_ERR_WORKSPACE;

@@ -267,10 +267,19 @@ __global__ void __launch_bounds__(kPfThreads, 2) prefill_chunk_kernel(PrefillPar
         // ---- O += P V ----
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk) {
-            const uint32_t a0 = pack_16x2<F16>(s[2 * kk][0], s[2 * kk][1]);
-            const uint32_t a1 = pack_16x2<F16>(s[2 * kk][2], s[2 * kk][3]);
-            const uint32_t a2 = pack_16x2<F16>(s[2 * kk + 1][0], s[2 * kk + 1][1]);
-            const uint32_t a3 = pack_16x2<F16>(s[2 * kk + 1][2], s[2 * kk + 1][3]);
+            // P enters the product as hi + lo, both 16-bit: hi = the rounded probability, lo = its rounding
+            // residual (exact in fp32). With the one-term product the residuals of the few probabilities that
+            // dominate a row are what is left of the output error (up to 5e-3 absolute with bf16).
+            uint32_t a[4], lo[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float p0 = s[2 * kk + (i >> 1)][2 * (i & 1)], p1 = s[2 * kk + (i >> 1)][2 * (i & 1) + 1];
+                float h0, h1;
+                a[i] = pack_16x2<F16>(p0, p1);
+                unpack_16x2<F16>(a[i], h0, h1);
+                lo[i] = pack_16x2<F16>(p0 - h0, p1 - h1);
+            }
+            const uint32_t a0 = a[0], a1 = a[1], a2 = a[2], a3 = a[3];
 #pragma unroll
             for (int dp = 0; dp < NT / 2; ++dp) {
                 const int mi = lane >> 3, rr = lane & 7;
@@ -280,6 +289,10 @@ __global__ void __launch_bounds__(kPfThreads, 2) prefill_chunk_kernel(PrefillPar
                 mma_16816<F16>(o[2 * dp][0], o[2 * dp][1], o[2 * dp][2], o[2 * dp][3], a0, a1, a2, a3, b0, b1,
                           o[2 * dp][0], o[2 * dp][1], o[2 * dp][2], o[2 * dp][3]);
                 mma_16816<F16>(o[2 * dp + 1][0], o[2 * dp + 1][1], o[2 * dp + 1][2], o[2 * dp + 1][3], a0, a1, a2, a3, b2, b3,
+                          o[2 * dp + 1][0], o[2 * dp + 1][1], o[2 * dp + 1][2], o[2 * dp + 1][3]);
+                mma_16816<F16>(o[2 * dp][0], o[2 * dp][1], o[2 * dp][2], o[2 * dp][3], lo[0], lo[1], lo[2], lo[3], b0, b1,
+                          o[2 * dp][0], o[2 * dp][1], o[2 * dp][2], o[2 * dp][3]);
+                mma_16816<F16>(o[2 * dp + 1][0], o[2 * dp + 1][1], o[2 * dp + 1][2], o[2 * dp + 1][3], lo[0], lo[1], lo[2], lo[3], b2, b3,
                           o[2 * dp + 1][0], o[2 * dp + 1][1], o[2 * dp + 1][2], o[2 * dp + 1][3]);
             }
         }

@@ -863,15 +863,7 @@ static int make_page_map(CUtensorMap *map, const void *layer_base, int num_block
     return rc == CUDA_SUCCESS ? EKV_OK : EKV_ERR_CUDA;
 }
 
-static int sm_count()
-{
-    static int n = [] {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) v = 0;
-        return v;
-    }();
-    return n;
-}
+static int sm_count() { return device_sm_count(); }
 
 // Workspace that lets the kernel balance its last wave: at most one piece per SM.
 size_t prefill_ws_workspace_bytes()

@@ -33,39 +33,70 @@ class ElasticRuntime:
         self.v_backing = torch.zeros(shape, dtype=torch.uint8).pin_memory()
         self.side = torch.cuda.Stream(device=dev)
         self.rows = {}                  # request id -> row of the device table
+        self.free_rows = list(range(max_batch - 1, -1, -1))
         self.lens = {}
+        self.boundaries = torch.zeros((max_batch, 2), dtype=torch.int32, device=dev)
+        self.flags = torch.zeros(4, dtype=torch.int32, device=dev)
         self.stats = {"demoted": 0, "promoted": 0}
 
     # ---- requests ----
-    def _sync_row(self, req):
-        t = self.ctrl.block_table(req)
-        row = self.rows[req]
-        self.block_table[row, : len(t)] = torch.from_numpy(t).to(self.block_table.device)
-        self.seq_lens[row] = self.lens[req]
+    def lower(self, reqs=None):
+        """Bring the device metadata of `reqs` (default: every live request) in line with the
+        controller: ONE host-to-device copy of the sparse description (lengths, block lists, BASE
+        pair ranges) and ONE library call that writes the table rows, the lengths, the structured
+        path's boundaries and the batch flags, and checks the ranges against the tags. Returns the
+        flags as a device tensor [any BASE, any irregular, disagreeing pairs, n - first such]."""
+        reqs = [r for r in (self.rows if reqs is None else reqs) if self.lens.get(r, 0) > 0]
+        lists = [self.ctrl.block_table(r) for r in reqs]
+        ranges = []
+        for r, t in zip(reqs, lists):
+            rr, start = [], None
+            for p in range(len(t) // 2 + 1):
+                is_base = p < len(t) // 2 and self.ctrl.pair_mode(r, p) == 1
+                if is_base and start is None:
+                    start = p
+                if not is_base and start is not None:
+                    rr += [start, p]
+                    start = None
+            ranges.append(rr)
+        parts = [np.array([self.rows[r] for r in reqs], np.int32), np.array([self.lens[r] for r in reqs], np.int32),
+                 np.concatenate([[0], np.cumsum([len(t) for t in lists])]).astype(np.int32),
+                 np.concatenate(lists).astype(np.int32) if lists else np.zeros(0, np.int32),
+                 np.concatenate([[0], np.cumsum([len(x) // 2 for x in ranges])]).astype(np.int32),
+                 np.array([v for x in ranges for v in x], np.int32)]
+        offs = np.concatenate([[0], np.cumsum([len(x) for x in parts])])
+        arena = torch.from_numpy(np.concatenate(parts).astype(np.int32)).to(self.block_table.device)
+        v = [arena[offs[k]:offs[k + 1]] for k in range(6)]
+        b.ekv_lower_sparse_metadata(self.pool, self.batch, self.seq_lens, v[0], v[1], v[2], v[3], v[4],
+                                    v[5] if len(v[5]) else None, self.boundaries, self.flags)
+        return self.flags
 
     def add_request(self, req, n_tokens):
         self.ctrl.add_request(req, n_tokens)
-        self.rows[req] = len(self.rows)
+        self.rows[req] = self.free_rows.pop()
         self.lens[req] = n_tokens
-        self._sync_row(req)
+        self.lower([req])
 
     def grow_request(self, req, n_tokens):
         self.ctrl.grow_request(req, n_tokens)
         self.lens[req] = n_tokens
-        self._sync_row(req)
+        self.lower([req])
 
     def finish_request(self, req):
-        """The request leaves: its blocks (and residual slots) return to the controller. Blocks that
-        stored a BASE pair are tagged TARGET again, since a released block carries no fidelity."""
+        """The request leaves: its blocks (and residual slots) return to the controller and its table
+        row to the free rows. Blocks that stored a BASE pair are tagged TARGET again (by the
+        library), since a released block carries no fidelity."""
         t = self.ctrl.block_table(req)
         base_blocks = [int(t[2 * p]) for p in range(len(t) // 2) if self.ctrl.pair_mode(req, p) == 1]
         self.ctrl.remove_request(req)
-        row = self.rows[req]
+        row = self.rows.pop(req)
         if base_blocks:
-            self.pool.tags[torch.tensor(base_blocks, device=self.pool.tags.device)] = 0
+            b.ekv_reset_tags(self.pool, self._dev(base_blocks))
         self.block_table[row] = -1
         self.seq_lens[row] = 0
-        self.lens[req] = 0
+        self.boundaries[row] = 0
+        del self.lens[req]
+        self.free_rows.append(row)
         return base_blocks
 
     def _dev(self, a):

@@ -128,3 +128,49 @@ def test_commit_rules_and_errors():
     freed = [int(c.block_table(7)[2 * p + 1]) for p in pi]
     c.commit_demotion(freed)
     assert c.last_surplus == 1
+
+
+def test_reserve_bounds_decay_and_budget():
+    """Properties Alg. 1 / Sec. 3.3 fix, checked on the controller alone with hand-computed numbers
+    (B_min = 6, lambda = 2, 40 blocks, one request of 30 blocks -> 10 free):
+      step 1: demand 12 -> Delta = 2, n_d = max(2, 6) = 6 <= eligible, E = 4, R_1 = 0 + 4 >= E, F_post = 16
+      then idle steps: R decays 4 -> 2 -> 0 in ceil(4 / 2) = 2 steps and stays 0;
+      the promotion budget is P_t = max(0, F_post - R_t) at every step (no transfer slack is granted,
+      so nothing is promoted and F_post stays 16)."""
+    c = controller.Controller(40, min_demote_pairs=6, reserve_decay=2, sink_pairs=0, recent_pairs=0, resid_slots=16)
+    c.add_request(1, 16 * 30)
+    assert c.free_blocks == 10
+    pr, pi, sl = c.plan_demotion(12)
+    assert c.last_shortage == 2 and len(pr) == 6           # Delta <= n_d <= |P_d|, n_d >= min(B_min, |P_d|)
+    c.commit_demotion([int(c.block_table(1)[2 * p + 1]) for p in pi])
+    assert c.last_surplus == 4 and c.free_blocks == 16
+    expected = [(4, 12), (2, 14), (0, 16), (0, 16)]        # (R_t, P_t) for steps 1..4
+    for t, (R, P) in enumerate(expected):
+        if t > 0:
+            assert len(c.plan_demotion(0)[0]) == 0
+        got = c.plan_promotion(0)
+        assert len(got[0]) == 0
+        assert (c.reserve, c.last_budget) == (R, P), f"step {t + 1}"
+        assert c.reserve >= (4 if t == 0 else 0)           # R_t >= E_t
+
+
+def test_a_step_without_a_promotion_plan_still_updates_the_reserve_once():
+    """lambda = 1, B_min = 4. Step 1 demotes with E_1 = 3 and never asks for a promotion plan; its
+    update R_1 = max(0, 0 - 1) + 3 = 3 is applied when step 2 opens. Step 2 (no shortage) asks
+    twice: R_2 = max(0, 3 - 1) + 0 = 2 both times. Step 3 has neither a shortage nor a promotion
+    plan; step 4 then sees R_3 = 1 applied and computes R_4 = 0."""
+    c = controller.Controller(40, min_demote_pairs=4, reserve_decay=1, sink_pairs=0, recent_pairs=0, resid_slots=16)
+    c.add_request(1, 16 * 30)
+    pr, pi, sl = c.plan_demotion(c.free_blocks + 1)
+    assert len(pr) == 4
+    c.commit_demotion([int(c.block_table(1)[2 * p + 1]) for p in pi])
+    assert c.last_surplus == 3
+    c.plan_demotion(0)                                     # step 2 opens
+    c.plan_promotion(0)
+    assert c.reserve == 2
+    c.plan_promotion(0)
+    assert c.reserve == 2                                  # once per step
+    c.plan_demotion(0)                                     # step 3: no promotion plan at all
+    c.plan_demotion(0)                                     # step 4
+    c.plan_promotion(0)
+    assert c.reserve == 0

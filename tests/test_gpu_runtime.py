@@ -80,6 +80,9 @@ def test_pressure_loop_with_controller(oracle):
         assert np.array_equal(rt.block_table.cpu().numpy(), op.block_table), f"step {step}: table"
         assert np.array_equal(words(pool.k_pool), op.k_pool), f"step {step}: k_pool"
         assert np.array_equal(words(pool.v_pool), op.v_pool), f"step {step}: v_pool"
+        fl = rt.lower().cpu().tolist()                                  # re-lowering the controller's view changes nothing
+        assert fl[2] == 0 and fl[0] == int(rt.ctrl.base_pairs > 0), f"step {step}: sparse metadata vs tags {fl}"
+        assert np.array_equal(rt.block_table.cpu().numpy(), op.block_table), f"step {step}: table after lowering"
         for r in range(n_req):                                          # controller and device agree
             if lens[r] == 0:
                 continue
@@ -87,3 +90,23 @@ def test_pressure_loop_with_controller(oracle):
             assert np.array_equal(t, rt.block_table[r, : len(t)].cpu().numpy())
     assert saw_demotion and saw_promotion
     assert rt.stats["demoted"] - rt.stats["promoted"] - released_pairs == rt.ctrl.base_pairs == int(pool.tags.sum().item())
+
+
+def test_table_rows_are_reused():
+    """A finished request gives its table row back: more requests than rows can pass through."""
+    b = require_gpu()
+    from paper_2609_33536_b200.runtime import ElasticRuntime
+    H, D = 2, 64
+    k = torch.zeros((1, 64, H * 16 * D), dtype=torch.int16, device="cuda")
+    pool = b.Pool(k, k.clone(), torch.zeros(64, dtype=torch.uint8, device="cuda"), H, D)
+    rt = ElasticRuntime(pool, max_batch=3, max_blocks=8, resid_slots=4)
+    for req in range(3):
+        rt.add_request(req, 40 + req)
+    for req in range(3, 9):
+        rt.finish_request(req - 3)
+        rt.add_request(req, 17 + req)
+        row = rt.rows[req]
+        assert 0 <= row < 3 and int(rt.seq_lens[row].item()) == 17 + req
+        t = rt.ctrl.block_table(req)
+        assert np.array_equal(rt.block_table[row, : len(t)].cpu().numpy(), t)
+    assert sorted(rt.rows.values()) == [0, 1, 2]

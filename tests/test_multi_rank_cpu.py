@@ -50,3 +50,19 @@ def test_single_process_is_identity():
     sys.path.insert(0, ROOT)
     import bench
     assert bench.aggregate_over_ranks(3.5, 7.0) == (3.5, 7.0)
+
+
+def test_bench_main_launches_its_own_ranks():
+    """`python bench.py --gpus 2` without a launcher around it starts its two ranks itself; driven
+    here through main() on CPU (gloo) with the kernels left out. Rank 0 alone prints the line."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    code = "import sys; sys.path.insert(0, %r); import bench; bench.main(['--gpus', '2', '--plumbing-check'])" % ROOT
+    out = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=240)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [ln for ln in out.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, out.stdout
+    res = json.loads(lines[0])
+    assert res["n_gpus"] == 2 and res["ms_per_step"] == 2.0          # the slower rank's time
+    assert res["bytes_all_ranks"] > res["bytes_rank0"] > 0           # both replicas' bytes
