@@ -113,6 +113,11 @@ const char *ekv_status_string(int status);
  *   "prefill_variant"     : 0 (default) = warp-specialised tcgen05 tensor-core kernel at
  *                           head_dim 128, mma.sync kernel otherwise; 1 = always the mma.sync
  *                           kernel (comparator).
+ *   "prefill_p_terms"     : how many 16-bit terms a probability enters the PV product of the tcgen05 prefill
+ *                           kernel with: 0 (default) = two for bf16 pools (the rounded value and its rounding
+ *                           residual; the residual costs a second pass of PV MMAs), one for fp16 pools;
+ *                           1 = one (faster; with bf16 the output's error before its final rounding can
+ *                           reach 5e-3 on rows that two or three tokens dominate); 2 = two.
  *   "decode_two_term"     : how the decode kernels treat the 16-bit rounding of the probabilities that
  *                           enter the PV product: 0 (default) = a step that holds a token with an eighth
  *                           or more of the probability mass its warp has seen so far takes PV a second

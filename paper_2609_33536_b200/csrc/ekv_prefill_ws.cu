@@ -255,7 +255,7 @@ __device__ __forceinline__ uint32_t ws_tile_off(int row, int ch16)
     return (uint32_t)((ch16 >> 3) * kWsHalf + row * 128 + (((ch16 & 7) ^ (row & 7)) << 4));
 }
 
-template <bool HAS_BASE, bool F16>
+template <bool HAS_BASE, bool F16, bool TWO_TERM, bool OUT_F32 = false>
 __global__ void __launch_bounds__(kWsThreads, 1) prefill_ws_kernel(PrefillTcParams p, const __grid_constant__ CUtensorMap map_k,
                                                                    const __grid_constant__ CUtensorMap map_v)
 {
@@ -427,13 +427,17 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_ws_kernel(PrefillTcPara
                 static_assert(kWsCols == 32, "one 32-column tensor-memory load per thread and tile");
                 const uint64_t scale2 = ws_pack2(p.scale_log2, p.scale_log2);
                 uint32_t pw[16];
+                uint32_t pl[TWO_TERM ? 16 : 1];           // two-term mode: the rounding residuals p - hi, as 16-bit pairs like pw
                 float tile_sum;
-                // P = 2^(s * scale - m) as packed 16-bit pairs over the scores; the row sum uses the rounded values (bf16) or the fp32 ones (fp16)
+                // P = 2^(s * scale - m) as packed 16-bit pairs over the scores. One-term mode: the row sum uses the
+                // rounded values (bf16) or the fp32 ones (fp16). Two-term mode: P enters the PV product as hi + lo,
+                // hi = the rounded probability, lo = its rounding residual (exact in fp32, then rounded to 16 bits
+                // itself: 2^-17 relative to p), and the sum takes the fp32 values.
                 auto exponentials = [&](float m) {
                     const float neg_m = m == -INFINITY ? 0.f : -m;
                     const uint64_t neg_m2 = ws_pack2(neg_m, neg_m);
-                    uint64_t sum2[2] = {0ull, 0ull};      // {even columns, odd columns} x 2 chains (fp16 pools)
-                    float sum1[2][2] = {{0.f, 0.f}, {0.f, 0.f}};              // the same four chains (bf16 pools)
+                    uint64_t sum2[2] = {0ull, 0ull};      // {even columns, odd columns} x 2 chains (fp32 sums)
+                    float sum1[2][2] = {{0.f, 0.f}, {0.f, 0.f}};              // the same four chains (sums of the rounded bf16 values)
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
                         const float s0 = __uint_as_float(sc[0][2 * i]), s1 = __uint_as_float(sc[0][2 * i + 1]);
@@ -441,15 +445,24 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_ws_kernel(PrefillTcPara
                         ws_unpack2(ws_fma2(ws_pack2(s0, s1), scale2, neg_m2), x0, x1);
                         const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
                         pw[i] = pack_16x2<F16>(p0, p1);
-                        // bf16: the sum has to see the rounding that P enters the PV product with (2^-9 relative on
-                        // a row that a few tokens dominate, next to the half-ulp of a bf16 output, breaks the 1e-2
-                        // bound); fp16 rounds eight times finer and takes the fp32 values as they are.
-                        // The bf16 halves go into the fp32 sums as they are (mixed-precision add): no unpacking.
-                        if (F16) sum2[i & 1] = ws_add2(sum2[i & 1], ws_pack2(p0, p1));
-                        else ws_add_bf16x2(sum1[i & 1][0], sum1[i & 1][1], pw[i]);
+                        if (TWO_TERM) {
+                            float h0, h1, l0, l1;
+                            unpack_16x2<F16>(pw[i], h0, h1);
+                            const uint64_t p2 = ws_pack2(p0, p1);
+                            ws_unpack2(ws_fma2(ws_pack2(h0, h1), ws_pack2(-1.f, -1.f), p2), l0, l1);
+                            pl[i] = pack_16x2<F16>(l0, l1);
+                            sum2[i & 1] = ws_add2(sum2[i & 1], p2);
+                        } else if (F16) {
+                            // fp16 rounds eight times finer than bf16 and takes the fp32 values as they are
+                            sum2[i & 1] = ws_add2(sum2[i & 1], ws_pack2(p0, p1));
+                        } else {
+                            // bf16, one term: the sum has to see the rounding that P enters the PV product with; the
+                            // bf16 halves go into the fp32 sums as they are (mixed-precision add): no unpacking
+                            ws_add_bf16x2(sum1[i & 1][0], sum1[i & 1][1], pw[i]);
+                        }
                     }
                     float e0 = sum1[0][0], o0 = sum1[0][1], e1 = sum1[1][0], o1 = sum1[1][1];
-                    if (F16) {
+                    if (F16 || TWO_TERM) {
                         ws_unpack2(sum2[0], e0, o0);
                         ws_unpack2(sum2[1], e1, o1);
                     }
@@ -510,6 +523,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_ws_kernel(PrefillTcPara
                     exponentials(m_ref[w]);
                 }
                 ws_st16(tmem_p, pw);
+                if (TWO_TERM) ws_st16(tmem_p + 64, (const uint32_t (&)[16])pl);     // the upper half of the score columns is free by now
                 l_run[w] += tile_sum;
                 ws_wait_st();
                 ws_fence_before();
@@ -546,7 +560,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_ws_kernel(PrefillTcPara
                     uint32_t v[32];
                     ws_ld32(tmem_o + q * 32, v);
                     ws_wait_ld();
-                    if (row_ok && p.out_f32) {
+                    if (OUT_F32 && row_ok) {
                         float *dstf = (float *)p.out + ((int64_t)(qs + row_i[w]) * p.num_q_heads + (g * G + row % Gp)) * kWsD + hf * kWsCols + q * 32;
 #pragma unroll
                         for (int c4 = 0; c4 < 8; ++c4) {
@@ -647,7 +661,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_ws_kernel(PrefillTcPara
                                 }
                             }
                         }
-                        if (row_ok && p.out_f32) {
+                        if (OUT_F32 && row_ok) {
                             float *dstf = (float *)p.out + ((int64_t)(qs + row_i[w]) * p.num_q_heads + (g * G + row % Gp)) * kWsD + hf * kWsCols + q * 32;
 #pragma unroll
                             for (int c4 = 0; c4 < 8; ++c4) {
@@ -793,6 +807,11 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_ws_kernel(PrefillTcPara
 #pragma unroll
             for (int k16 = 0; k16 < kWsKv / 16; ++k16)
                 ws_mma_ts(d, a + (uint32_t)(8 * k16), vb + (uint32_t)((k16 * 2048) >> 4), kIdescPV, (j > 0) || (k16 > 0), leader);
+            if (TWO_TERM) {                               // the residual terms of P, 64 columns further on
+#pragma unroll
+                for (int k16 = 0; k16 < kWsKv / 16; ++k16)
+                    ws_mma_ts(d, a + (uint32_t)(64 + 8 * k16), vb + (uint32_t)((k16 * 2048) >> 4), kIdescPV, 1u, leader);
+            }
         };
         if (n_tiles > 0) {
             wait(kBarKFull + 0, 0u);                      // Q and K(0)
@@ -906,22 +925,46 @@ int launch_prefill_ws(const PrefillTcParams &p_in, int64_t ctas, int max_pages, 
             if (cudaMemsetAsync(p.part_count, 0, (size_t)rem * sizeof(int), st) != cudaSuccess) return EKV_ERR_CUDA;
         }
     }
-    cudaError_t err;
-    if (has_base) {
-        err = f16 ? cudaFuncSetAttribute(prefill_ws_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm)
-                  : cudaFuncSetAttribute(prefill_ws_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-        if (err != cudaSuccess) return EKV_ERR_CUDA;
-        MainKernelScope scope(st);
-        if (f16) prefill_ws_kernel<true, true><<<(unsigned)grid, kWsThreads, sm, st>>>(p, map_k, map_v);
-        else prefill_ws_kernel<true, false><<<(unsigned)grid, kWsThreads, sm, st>>>(p, map_k, map_v);
+    // Probabilities enter the PV product as one 16-bit term, or as two (rounded value + rounding residual).
+    // Default: two for bf16 pools (one bf16 term leaves up to 5e-3 of output error on rows that a few tokens
+    // dominate), one for fp16 pools (eight times finer); "prefill_p_terms" overrides.
+    const bool two = g_prefill_p_terms == 0 ? !f16 : g_prefill_p_terms == 2;
+    cudaError_t err = cudaSuccess;
+#define EKV_LAUNCH_WS(HB, FF, TT)                                                                          \
+    do {                                                                                                  \
+        err = cudaFuncSetAttribute(prefill_ws_kernel<HB, FF, TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm); \
+        if (err == cudaSuccess) {                                                                         \
+            MainKernelScope scope(st);                                                                    \
+            prefill_ws_kernel<HB, FF, TT><<<(unsigned)grid, kWsThreads, sm, st>>>(p, map_k, map_v);       \
+        }                                                                                                 \
+    } while (0)
+    if (p.out_f32) {
+        // debug output in fp32: its own instantiations, so that the production kernels carry no trace of it
+#define EKV_LAUNCH_WS_F32(HB, FF, TT)                                                                      \
+    do {                                                                                                  \
+        err = cudaFuncSetAttribute(prefill_ws_kernel<HB, FF, TT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm); \
+        if (err == cudaSuccess) {                                                                         \
+            MainKernelScope scope(st);                                                                    \
+            prefill_ws_kernel<HB, FF, TT, true><<<(unsigned)grid, kWsThreads, sm, st>>>(p, map_k, map_v); \
+        }                                                                                                 \
+    } while (0)
+        if (has_base) {
+            if (f16) { if (two) EKV_LAUNCH_WS_F32(true, true, true); else EKV_LAUNCH_WS_F32(true, true, false); }
+            else     { if (two) EKV_LAUNCH_WS_F32(true, false, true); else EKV_LAUNCH_WS_F32(true, false, false); }
+        } else {
+            if (f16) { if (two) EKV_LAUNCH_WS_F32(false, true, true); else EKV_LAUNCH_WS_F32(false, true, false); }
+            else     { if (two) EKV_LAUNCH_WS_F32(false, false, true); else EKV_LAUNCH_WS_F32(false, false, false); }
+        }
+#undef EKV_LAUNCH_WS_F32
+    } else if (has_base) {
+        if (f16) { if (two) EKV_LAUNCH_WS(true, true, true); else EKV_LAUNCH_WS(true, true, false); }
+        else     { if (two) EKV_LAUNCH_WS(true, false, true); else EKV_LAUNCH_WS(true, false, false); }
     } else {
-        err = f16 ? cudaFuncSetAttribute(prefill_ws_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm)
-                  : cudaFuncSetAttribute(prefill_ws_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-        if (err != cudaSuccess) return EKV_ERR_CUDA;
-        MainKernelScope scope(st);
-        if (f16) prefill_ws_kernel<false, true><<<(unsigned)grid, kWsThreads, sm, st>>>(p, map_k, map_v);
-        else prefill_ws_kernel<false, false><<<(unsigned)grid, kWsThreads, sm, st>>>(p, map_k, map_v);
+        if (f16) { if (two) EKV_LAUNCH_WS(false, true, true); else EKV_LAUNCH_WS(false, true, false); }
+        else     { if (two) EKV_LAUNCH_WS(false, false, true); else EKV_LAUNCH_WS(false, false, false); }
     }
+#undef EKV_LAUNCH_WS
+    if (err != cudaSuccess) return EKV_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? EKV_OK : EKV_ERR_CUDA;
 }
 
