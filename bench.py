@@ -522,6 +522,81 @@ def transitions_multi_layer(b, torch, dev, i32, flush, num_layers):
             "downgrade": {"us": round(float(np.median(td)) * 1e3, 1), "GBps": round(down_b / np.median(td) / 1e6, 1)},
             "refine": {"us": round(float(np.median(tu)) * 1e3, 1), "GBps": round(up_b / np.median(tu) / 1e6, 1)}}
 
+def metadata_lowering(b, torch, dev, batch=256):
+    """Worker-side metadata lowering for one step of the high-concurrency configuration: the scheduler's
+    sparse description (lengths, block lists, BASE pair ranges of all 256 requests) goes up in ONE pinned
+    host-to-device copy and ekv_lower_sparse_metadata writes table rows, lengths, boundaries and flags in
+    one launch; beside it, the same update done request by request with torch copies (one table-row copy
+    and one length write per request). Host wall clock per step, device synchronised at the end."""
+    wl = synth.cfg_pressure()
+    pool, bt, q = b.upload(wl, dev)
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+    fr = torch.empty(len(wl.base_pair_req), dtype=torch.int32, device=dev)
+    b.ekv_downgrade(pool, bt, i32(wl.base_pair_req), i32(wl.base_pair_idx), None, None, None, fr)
+    torch.cuda.synchronize()
+    table = bt.block_table.cpu().numpy()
+    tags = pool.tags.cpu().numpy()
+    lists, ranges = [], []
+    for r in range(wl.batch):
+        nb = -(-int(wl.seq_lens[r]) // wl.page_size)
+        ids = table[r, :nb]
+        lists.append(ids)
+        base = tags[ids[0::2]] == 1
+        rr, start = [], None
+        for pidx, flag in enumerate(list(base) + [False]):
+            if flag and start is None:
+                start = pidx
+            if not flag and start is not None:
+                rr += [start, pidx]; start = None
+        ranges.append(rr)
+    parts = [np.arange(wl.batch, dtype=np.int32), wl.seq_lens.astype(np.int32),
+             np.concatenate([[0], np.cumsum([len(x) for x in lists])]).astype(np.int32), np.concatenate(lists).astype(np.int32),
+             np.concatenate([[0], np.cumsum([len(x) // 2 for x in ranges])]).astype(np.int32),
+             np.array([v for x in ranges for v in x], np.int32)]
+    offs = np.concatenate([[0], np.cumsum([len(x) for x in parts])])
+    arena_h = torch.from_numpy(np.concatenate(parts).astype(np.int32)).pin_memory()
+    arena_d = torch.empty_like(arena_h, device=dev)
+    v = [arena_d[offs[k]:offs[k + 1]] for k in range(6)]
+    out_table = torch.full_like(bt.block_table, -1)
+    out_sl = torch.zeros_like(bt.seq_lens)
+    out_batch = b.Batch(out_table, out_sl, True)
+    bounds = torch.zeros((wl.batch, 2), dtype=torch.int32, device=dev)
+    flags = torch.zeros(4, dtype=torch.int32, device=dev)
+
+    def lowered():
+        arena_d.copy_(arena_h, non_blocking=True)
+        b.ekv_lower_sparse_metadata(pool, out_batch, out_sl, v[0], v[1], v[2], v[3], v[4], v[5] if len(v[5]) else None, bounds, flags)
+        torch.cuda.synchronize()
+
+    host_rows = [torch.from_numpy(np.ascontiguousarray(x)).pin_memory() for x in lists]
+    lens_h = wl.seq_lens.tolist()
+
+    def per_request():
+        for r in range(wl.batch):
+            out_table[r, : len(lists[r])].copy_(host_rows[r], non_blocking=True)
+            out_sl[r] = lens_h[r]
+        torch.cuda.synchronize()
+
+    def wall(fn, n=20):
+        for _ in range(3):
+            fn()
+        t0 = time.perf_counter()
+        for _ in range(n):
+            fn()
+        return (time.perf_counter() - t0) / n
+    t_low = wall(lowered)
+    assert torch.equal(out_table[:, :1], bt.block_table[:, :1]) and flags.cpu().tolist()[2] == 0
+    t_py = wall(per_request, n=5)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(20):
+        b.ekv_lower_sparse_metadata(pool, out_batch, out_sl, v[0], v[1], v[2], v[3], v[4], v[5] if len(v[5]) else None, bounds, flags)
+    e1.record(); torch.cuda.synchronize()
+    return {"workload": f"batch {wl.batch} of the high-concurrency configuration, {int(offs[-1]) * 4} bytes of sparse description",
+            "lowered_us_per_step": round(t_low * 1e6, 1), "kernel_us": round(e0.elapsed_time(e1) / 20 * 1e3, 2),
+            "per_request_copies_us_per_step": round(t_py * 1e6, 1), "flags": flags.cpu().tolist()}
+
+
 def extras(b, torch, dev, args):
     """Context numbers (not part of the timed step): decode GB/s over the BASE-fraction sweep,
     the native / elastic-idle comparison on the all-TARGET pool, and transition GB/s."""
@@ -699,8 +774,12 @@ def extras(b, torch, dev, args):
     C, L = int(wl.q_start[1]), int(wl.seq_lens[0])
     flops = 4.0 * wl.head_dim * wl.num_q_heads * sum(L - C + i + 1 for i in range(C)) * wl.batch
     pf_ws = b.new_workspace(pool, wl.batch, wl.num_q_heads, L, int(wl.q_start[-1]))
-    ms = timed(lambda: b.ekv_attn_prefill_chunk(pool, 0, batch, qs, q, out, wl.num_q_heads, wl.sm_scale,
-                                                int(wl.q_start[-1]), C, L, pf_ws), iters=10, warm=3)
+    run_pf = lambda: b.ekv_attn_prefill_chunk(pool, 0, batch, qs, q, out, wl.num_q_heads, wl.sm_scale,
+                                              int(wl.q_start[-1]), C, L, pf_ws)
+    ms = timed(run_pf, iters=10, warm=3)
+    b.ekv_set_option("prefill_p_terms", 1)                  # one bf16 term per probability: faster, outside the error bound on some rows
+    ms_one = timed(run_pf, iters=10, warm=3)
+    b.ekv_set_option("prefill_p_terms", 0)
     peak = 1609.8
     try:
         peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops"])
@@ -708,7 +787,15 @@ def extras(b, torch, dev, args):
         pass
     res["prefill_chunk"] = {"workload": "batch 8, 512-token chunk over an 8192-token prefix (50 % BASE), 32/8 heads, D 128",
                             "ms": round(ms, 4), "TFLOPs": round(flops / ms / 1e9, 1), "peak_TFLOPs": peak,
-                            "frac": round(flops / ms / 1e9 / peak, 4), "bound": "tensor"}
+                            "frac": round(flops / ms / 1e9 / peak, 4), "bound": "tensor",
+                            "p_terms": "two 16-bit terms per probability (default for bf16 pools)",
+                            "one_term": {"ms": round(ms_one, 4), "TFLOPs": round(flops / ms_one / 1e9, 1),
+                                         "frac": round(flops / ms_one / 1e9 / peak, 4),
+                                         "note": "option prefill_p_terms = 1: the output's error before its final rounding "
+                                                 "reaches 5e-3 on rows that two or three tokens dominate"}}
+    del pool, batch, q, out, pf_ws
+    torch.cuda.empty_cache()
+    res["metadata_lowering"] = metadata_lowering(b, torch, dev)
     return res
 
 
@@ -757,6 +844,12 @@ def roofline_others(ex, hbm_peak):
                         "frac_of_sustained": round(pf["TFLOPs"] / tf_sust, 4), "us": round(pf["ms"] * 1e3, 1),
                         "workload": "chunked prefill: batch 8, 512-token chunk over an 8192-token prefix (50 % BASE), 32/8 heads, D 128; "
                                     "L2 flushed before every launch"})
+    pf1 = ex.get("prefill_chunk", {}).get("one_term")
+    if pf1:
+        out.append({"kernel": "prefill_ws_kernel (bf16, option prefill_p_terms = 1: one term per probability)", "bound": "tensor",
+                    "achieved": pf1["TFLOPs"], "peak": tf_burst, "unit": "TFLOP/s", "frac": round(pf1["TFLOPs"] / tf_burst, 4),
+                    "peak_sustained": tf_sust, "frac_of_sustained": round(pf1["TFLOPs"] / tf_sust, 4), "us": round(pf1["ms"] * 1e3, 1),
+                    "workload": "the same chunked-prefill configuration"})
     return out
 
 

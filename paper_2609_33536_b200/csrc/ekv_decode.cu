@@ -1054,16 +1054,31 @@ static cudaError_t launch_merge(const DecodeParams &p, int rows, cudaStream_t st
     return cudaLaunchKernelEx(&cfg, decode_merge_kernel<D, F16, 1>, p);
 }
 
-// Tokens per split. Automatic choice: enough CTAs for about six waves of 3 CTAs per SM when every
-// sequence has the maximum length, clamped to [256, 4096] and rounded to 64 tokens.
+// Tokens per split. Automatic choice, from the upper bound max_seq_len of every sequence:
+//   - small launches (all units = requests x kv heads fit, with splits of at most 4096 tokens, into two
+//     CTAs per SM): as many equal splits per unit as keep the grid within two CTAs per SM, i.e. one
+//     balanced wave; more, smaller CTAs only add per-CTA set-up and a merge with more partials;
+//   - otherwise: about three waves of 3 CTAs per SM, at most 3200 tokens (large splits pay in the last
+//     wave, where an SM left with one CTA cannot draw its share of the bandwidth), at least 256.
+// Rounded to 64 tokens so that a pair never straddles splits.
 int decode_chunk_tokens(int batch, int num_kv_heads, int max_seq_len)
 {
     int64_t chunk = g_decode_chunk_tokens;
     if (chunk <= 0) {
-        const int64_t want_ctas = (int64_t)device_sm_count() * 3 * 6;
-        chunk = ((int64_t)max_seq_len * batch * num_kv_heads + want_ctas - 1) / want_ctas;
+        const int64_t sms = device_sm_count();
+        const int64_t units = (int64_t)batch * num_kv_heads;
+        const int64_t len = max_seq_len > 0 ? max_seq_len : 1;
+        if (units * ((len + kMaxChunkTokens - 1) / kMaxChunkTokens) <= 2 * sms) {
+            int64_t splits = 2 * sms / units;
+            if (splits > (len + 255) / 256) splits = (len + 255) / 256;
+            if (splits < 1) splits = 1;
+            chunk = (len + splits - 1) / splits;
+        } else {
+            const int64_t want_ctas = sms * 3 * 3;
+            chunk = (len * units + want_ctas - 1) / want_ctas;
+            if (chunk > 3200) chunk = 3200;
+        }
         if (chunk < 256) chunk = 256;
-        if (chunk > kMaxChunkTokens) chunk = kMaxChunkTokens;
     }
     if (chunk > kMaxChunkTokens) chunk = kMaxChunkTokens;      // a warp's step list holds 32 pairs
     chunk = (chunk + 63) / 64 * 64;
