@@ -459,7 +459,7 @@ __device__ __forceinline__ void softmax_step_t(float (&s)[MTILES][4], int valid,
     // the masked scores are parked in this lane's shared-memory slot: the rare two-term pass takes them from there
 #pragma unroll
     for (int mt = 0; mt < MTILES; ++mt)
-        asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" :: "r"(save_addr + 16 * mt), "f"(s[mt][0]), "f"(s[mt][1]), "f"(s[mt][2]), "f"(s[mt][3]) : "memory");
+        asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" :: "r"(save_addr + 512 * mt), "f"(s[mt][0]), "f"(s[mt][1]), "f"(s[mt][2]), "f"(s[mt][3]) : "memory");
     float mx[2];
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
@@ -502,7 +502,7 @@ __device__ __forceinline__ void two_term_residuals(uint32_t save_addr, const flo
 #pragma unroll
     for (int mt = 0; mt < MTILES; ++mt) {
         float s0, s1, s2, s3, h0, h1, h2, h3;
-        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(s0), "=f"(s1), "=f"(s2), "=f"(s3) : "r"(save_addr + 16 * mt) : "memory");
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(s0), "=f"(s1), "=f"(s2), "=f"(s3) : "r"(save_addr + 512 * mt) : "memory");
         const float p0 = fast_exp2(s0 - m_run[0]), p1 = fast_exp2(s1 - m_run[1]);
         const float p2 = fast_exp2(s2 - m_run[0]), p3 = fast_exp2(s3 - m_run[1]);
         unpack_16x2<F16>(pack_16x2<F16>(p0, p1), h0, h1);
@@ -579,10 +579,11 @@ __global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(D
     float (*sm_m)[8] = (float (*)[8])((uint8_t *)sm_q + KS * 32 * sizeof(uint2));
     float (*sm_l)[8] = sm_m + kDecodeWarps;
     uint2 *sm_steps = (uint2 *)(sm_l + kDecodeWarps);     // [4 warps][64] step descriptors
-    const uint32_t save_addr = (uint32_t)__cvta_generic_to_shared(sm_steps + kDecodeWarps * 64) + threadIdx.x * 32;   // this lane's parked scores of a step
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int c = lane >> 2, j = lane & 3;
+    // parked scores of a step: [warp][m-tile][lane] x 16 bytes, so that a warp's stores fall on consecutive banks
+    const uint32_t save_addr = (uint32_t)__cvta_generic_to_shared(sm_steps + kDecodeWarps * 64) + warp * 1024 + lane * 16;
 
     int idx = blockIdx.x;
     const int g = idx % p.num_kv_heads; idx /= p.num_kv_heads;

@@ -14,13 +14,13 @@ struct LowerParams {
     int n_req, max_blocks, num_blocks;
 };
 
-// One warp per scheduled request. Lanes walk the request's blocks (copy into its table row) and
+// One CTA per scheduled request. Threads walk the request's blocks (copy into its table row) and
 // its pairs (mode by binary search in the request's sorted ranges, compared with the tag).
-__global__ void lower_sparse_kernel(LowerParams p)
+constexpr int kLowerThreads = 128;
+__global__ void __launch_bounds__(kLowerThreads) lower_sparse_kernel(LowerParams p)
 {
-    const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (i >= p.n_req) return;
+    const int i = blockIdx.x;
+    const int tid = threadIdx.x;
     const int row = p.row_of ? p.row_of[i] : i;
     const int L = p.lens[i];
     const int b0 = p.blk_start[i], nb = p.blk_start[i + 1] - b0;
@@ -28,26 +28,17 @@ __global__ void lower_sparse_kernel(LowerParams p)
     const int32_t *ids = p.blk_ids + b0;
     const int32_t *rg = p.ranges + 2 * (int64_t)r0;
     int32_t *dst = p.block_table + (int64_t)row * p.max_blocks;
-    for (int lb = lane; lb < nb && lb < p.max_blocks; lb += 32) dst[lb] = ids[lb];
-    if (lane == 0) p.seq_lens[row] = L;
+    for (int lb = tid; lb < nb && lb < p.max_blocks; lb += kLowerThreads) dst[lb] = ids[lb];
 
-    // ranges -> boundaries and the regular / irregular verdict (sorted, disjoint; two ranges that touch count as one)
+    // ranges -> the regular / irregular verdict (sorted, disjoint; two ranges that touch count as one)
     int gaps = 0;
-    for (int k = lane + 1; k < nr; k += 32) gaps += rg[2 * k] > rg[2 * k - 1] ? 1 : 0;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) gaps += __shfl_xor_sync(0xffffffffu, gaps, o);
-    if (lane == 0) {
-        p.boundaries[2 * row] = nr > 0 ? rg[0] : 0;
-        p.boundaries[2 * row + 1] = nr > 0 ? rg[2 * nr - 1] : 0;
-        if (nr > 0) atomicOr(&p.flags[0], 1);
-        if (gaps > 0) atomicOr(&p.flags[1], 1);
-    }
+    for (int k = tid + 1; k < nr; k += kLowerThreads) gaps += rg[2 * k] > rg[2 * k - 1] ? 1 : 0;
 
     // cross-check against the tags: a pair is BASE exactly when it lies in a range, and then both of
     // its table entries name the one block that stores it
     const int npairs = (nb + 1) / 2;
     int bad = 0;
-    for (int pp = lane; pp < npairs; pp += 32) {
+    for (int pp = tid; pp < npairs; pp += kLowerThreads) {
         int lo = 0, hi = nr;                               // first range whose end is beyond pp
         while (lo < hi) { const int mid = (lo + hi) >> 1; if (rg[2 * mid + 1] > pp) hi = mid; else lo = mid + 1; }
         const bool in_range = lo < nr && rg[2 * lo] <= pp;
@@ -60,11 +51,22 @@ __global__ void lower_sparse_kernel(LowerParams p)
         }
         bad += ok ? 0 : 1;
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) bad += __shfl_xor_sync(0xffffffffu, bad, o);
-    if (lane == 0 && bad > 0) {
-        atomicAdd(&p.flags[2], bad);
-        atomicMax(&p.flags[3], p.n_req - i);             // largest for the first request; 0 = none
+    const int any_gap = __syncthreads_or(gaps);
+    __shared__ int sm_bad;
+    if (tid == 0) sm_bad = 0;
+    __syncthreads();
+    if (bad) atomicAdd(&sm_bad, bad);
+    __syncthreads();
+    if (tid == 0) {
+        p.seq_lens[row] = L;
+        p.boundaries[2 * row] = nr > 0 ? rg[0] : 0;
+        p.boundaries[2 * row + 1] = nr > 0 ? rg[2 * nr - 1] : 0;
+        if (nr > 0) atomicOr(&p.flags[0], 1);
+        if (any_gap) atomicOr(&p.flags[1], 1);
+        if (sm_bad > 0) {
+            atomicAdd(&p.flags[2], sm_bad);
+            atomicMax(&p.flags[3], p.n_req - i);           // largest for the first request; 0 = none
+        }
     }
 }
 
@@ -100,7 +102,7 @@ extern "C" int ekv_lower_sparse_metadata(const ekv_pool *pool, const ekv_batch *
         p.block_table = batch->block_table; p.seq_lens = seq_lens_out;
         p.boundaries = boundaries; p.flags = flags;
         p.n_req = n_req; p.max_blocks = batch->max_blocks; p.num_blocks = pool->num_blocks;
-        lower_sparse_kernel<<<(n_req + 3) / 4, 128, 0, st>>>(p);
+        lower_sparse_kernel<<<n_req, kLowerThreads, 0, st>>>(p);
     }
     return cudaGetLastError() == cudaSuccess ? EKV_OK : EKV_ERR_CUDA;
 }

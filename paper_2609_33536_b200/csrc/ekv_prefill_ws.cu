@@ -241,6 +241,19 @@ __device__ __forceinline__ void ws_add_bf16x2(float &lo, float &hi, uint32_t pw)
         "add.rn.f32.bf16 %0, hl, %0;\n\tadd.rn.f32.bf16 %1, hh, %1;\n\t}"
         : "+f"(lo), "+f"(hi) : "r"(pw));
 }
+// d0 = (low 16-bit half of pw) - c0, d1 = (high half) - c1: the halves widen exactly, the differences round to nearest in fp32
+template <bool F16>
+__device__ __forceinline__ void ws_sub_16x2(float &d0, float &d1, uint32_t pw, float c0, float c1)
+{
+    if (F16)
+        asm("{\n\t.reg .b16 hl, hh;\n\tmov.b32 {hl, hh}, %2;\n\t"
+            "sub.rn.f32.f16 %0, hl, %3;\n\tsub.rn.f32.f16 %1, hh, %4;\n\t}"
+            : "=f"(d0), "=f"(d1) : "r"(pw), "f"(c0), "f"(c1));
+    else
+        asm("{\n\t.reg .b16 hl, hh;\n\tmov.b32 {hl, hh}, %2;\n\t"
+            "sub.rn.f32.bf16 %0, hl, %3;\n\tsub.rn.f32.bf16 %1, hh, %4;\n\t}"
+            : "=f"(d0), "=f"(d1) : "r"(pw), "f"(c0), "f"(c1));
+}
 __device__ __forceinline__ float ws_max3(float a, float b, float c)
 {
     float d;
@@ -446,12 +459,12 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_ws_kernel(PrefillTcPara
                         const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
                         pw[i] = pack_16x2<F16>(p0, p1);
                         if (TWO_TERM) {
-                            float h0, h1, l0, l1;
-                            unpack_16x2<F16>(pw[i], h0, h1);
-                            const uint64_t p2 = ws_pack2(p0, p1);
-                            ws_unpack2(ws_fma2(ws_pack2(h0, h1), ws_pack2(-1.f, -1.f), p2), l0, l1);
-                            pl[i] = pack_16x2<F16>(l0, l1);
-                            sum2[i & 1] = ws_add2(sum2[i & 1], p2);
+                            // pl holds hi - p, the NEGATED residual: one mixed-precision subtract per element, no
+                            // unpacking; the instruction descriptor of the residual MMA negates A to match
+                            float n0, n1;
+                            ws_sub_16x2<F16>(n0, n1, pw[i], p0, p1);
+                            pl[i] = pack_16x2<F16>(n0, n1);
+                            sum2[i & 1] = ws_add2(sum2[i & 1], ws_pack2(p0, p1));
                         } else if (F16) {
                             // fp16 rounds eight times finer than bf16 and takes the fp32 values as they are
                             sum2[i & 1] = ws_add2(sum2[i & 1], ws_pack2(p0, p1));
@@ -807,10 +820,10 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_ws_kernel(PrefillTcPara
 #pragma unroll
             for (int k16 = 0; k16 < kWsKv / 16; ++k16)
                 ws_mma_ts(d, a + (uint32_t)(8 * k16), vb + (uint32_t)((k16 * 2048) >> 4), kIdescPV, (j > 0) || (k16 > 0), leader);
-            if (TWO_TERM) {                               // the residual terms of P, 64 columns further on
+            if (TWO_TERM) {                               // the residual terms of P (stored negated), 64 columns further on
 #pragma unroll
                 for (int k16 = 0; k16 < kWsKv / 16; ++k16)
-                    ws_mma_ts(d, a + (uint32_t)(64 + 8 * k16), vb + (uint32_t)((k16 * 2048) >> 4), kIdescPV, 1u, leader);
+                    ws_mma_ts(d, a + (uint32_t)(64 + 8 * k16), vb + (uint32_t)((k16 * 2048) >> 4), kIdescPV | (1u << 13), 1u, leader);   // bit 13: negate A
             }
         };
         if (n_tiles > 0) {

@@ -114,3 +114,39 @@ def test_recorded_prefill_offenders(oracle, case):
     that a few tokens dominate)."""
     b = require_gpu()
     run_case(b, oracle, case)
+
+
+def test_one_term_options_stay_close_to_the_default(oracle):
+    """The measurement options that switch the second probability term off (decode_two_term = 1,
+    prefill_p_terms = 1) or force it on (2) change results only at the level the second term is
+    there to remove: within 6e-3 of the oracle before the output rounding (one term), within the
+    pre-rounding bound (two terms)."""
+    b = require_gpu()
+    rs = np.random.default_rng(31)
+    for kind, opt, one, two in (("decode", "decode_two_term", 1, 2), ("prefill", "prefill_p_terms", 1, 2)):
+        for _ in range(12):
+            c = draw_case(rs, kind)
+            c["et"], c["v"] = "bf16", 0
+            kw = dict(seed=c["seed"], seq_lens=c["lens"], num_q_heads=c["G"] * c["H"], num_kv_heads=c["H"], head_dim=c["D"],
+                      base_fraction=c["f"], base_pattern=c["pat"], elem_type="bf16")
+            if kind == "decode":
+                wl = synth.make_workload("fz", **kw)
+                op, *_ = mixed_oracle_pool(oracle, wl)
+                exp = oracle.attn_decode(op, 0, wl.q, wl.num_q_heads, wl.sm_scale)
+                pool, batch, q = upload_state(b, op, wl.q)
+                run = lambda: gpu_decode(b, pool, batch, q, wl.num_q_heads, wl.sm_scale, f32=True)
+            else:
+                wl = synth.make_workload("fz", chunk_lens=c["chunks"], **kw)
+                op, *_ = mixed_oracle_pool(oracle, wl)
+                exp = oracle.attn_prefill_chunk(op, 0, wl.q_start, wl.q, wl.num_q_heads, wl.sm_scale)
+                pool, batch, q = upload_state(b, op, wl.q)
+                run = lambda: gpu_prefill(b, pool, batch, q, wl, f32=True)
+            try:
+                b.ekv_set_option(opt, one)
+                got1 = run()
+                b.ekv_set_option(opt, two)
+                got2 = run()
+            finally:
+                b.ekv_set_option(opt, 0)
+            assert np.abs(got1 - exp).max() <= 6e-3 * max(1.0, np.abs(exp).max() / 4), (kind, c)
+            assert_attn_close_f32(got2, exp, f"{opt} = {two}: {c}")
