@@ -118,6 +118,10 @@ const char *ekv_status_string(int status);
  *                           residual; the residual costs a second pass of PV MMAs), one for fp16 pools;
  *                           1 = one (faster; with bf16 the output's error before its final rounding can
  *                           reach 5e-3 on rows that two or three tokens dominate); 2 = two.
+ *   "decode_staging"      : how the ring-staged decode kernel brings K/V slabs into shared memory: 0 or 1
+ *                           (default) = cp.async, 16 bytes per lane and instruction; 2 = TMA tensor copies
+ *                           (head_dim 128 only; one lane issues two box copies per slab, completion on an
+ *                           mbarrier). Same results; measured 1-2 % slower, kept for measurements.
  *   "decode_two_term"     : how the decode kernels treat the 16-bit rounding of the probabilities that
  *                           enter the PV product: 0 (default) = a step that holds a token with an eighth
  *                           or more of the probability mass its warp has seen so far takes PV a second
@@ -278,6 +282,11 @@ int ekv_attn_prefill_chunk(const ekv_pool *pool, int32_t layer, const ekv_batch 
 int ekv_kv_append(const ekv_pool *pool, int32_t layer, const ekv_batch *batch, const int32_t *q_start,
                   const void *k_new, const void *v_new, int32_t total_new, int32_t *dev_status,
                   void *stream);
+
+/* Debug query for the TMA-staged decode kernel (no paper counterpart): synchronises the device, returns the
+ * kernel's status word and clears it: 0 = ok, 1 = a bounded wait for a staged slab expired (results are
+ * invalid); negative = ekv_status. */
+int ekv_decode_status(void);
 
 /* Debug query for the tensor-core prefill kernel (no paper counterpart). Synchronises the
  * device, returns the kernel's status word and clears it: 0 = ok, 1 = a bounded wait inside the

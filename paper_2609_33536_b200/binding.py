@@ -17,7 +17,7 @@ EXPORTS = ("ekv_version", "ekv_status_string", "ekv_set_option", "ekv_set_profil
            "ekv_attn_decode", "ekv_attn_prefill_chunk", "ekv_downgrade", "ekv_refine",
            "ekv_validate_batch", "ekv_attn_decode_noalloc", "ekv_attn_decode_noalloc_max_bytes",
            "ekv_prefill_status", "ekv_lower_metadata", "ekv_attn_decode_structured",
-           "ekv_kv_append", "ekv_lower_sparse_metadata", "ekv_reset_tags")
+           "ekv_kv_append", "ekv_lower_sparse_metadata", "ekv_reset_tags", "ekv_decode_status")
 
 
 class EkvError(RuntimeError):
@@ -85,6 +85,7 @@ def load(path: str | None = None):
         L.ekv_reset_tags.restype = C.c_int
         L.ekv_reset_tags.argtypes = [PP, vp, i32, vp]
         L.ekv_prefill_status.restype = C.c_int
+        L.ekv_decode_status.restype = C.c_int
         L.ekv_validate_batch.restype = C.c_int
         L.ekv_validate_batch.argtypes = [PP, BP, vp, vp]
         _lib = L
@@ -238,6 +239,11 @@ def ekv_kv_append(pool: Pool, layer: int, batch: Batch, q_start, k_new, v_new, d
     _check(load().ekv_kv_append(C.byref(pool.c), layer, C.byref(batch.c), _ptr(q_start), _ptr(k_new), _ptr(v_new),
                                 int(k_new.shape[0]), _ptr(dev_status), _stream()),
            "ekv_kv_append")
+
+
+def ekv_decode_status() -> int:
+    """Status word of the TMA-staged decode kernel (synchronises; 0 = ok); clears it."""
+    return int(load().ekv_decode_status())
 
 
 def ekv_prefill_status() -> int:

@@ -12,6 +12,7 @@ int64_t g_decode_merge_slices = 0;
 int64_t g_prefill_variant = 0;
 int64_t g_attn_out_f32 = 0;
 int64_t g_decode_two_term = 0;
+int64_t g_decode_staging = 0;
 int64_t g_prefill_p_terms = 0;
 void *g_profile_ev[2] = {nullptr, nullptr};
 
@@ -98,6 +99,11 @@ extern "C" int ekv_set_option(const char *name, int64_t value)
     if (!strcmp(name, "prefill_p_terms")) {
         if (value < 0 || value > 2) return EKV_ERR_INVALID_ARG;
         g_prefill_p_terms = value;
+        return EKV_OK;
+    }
+    if (!strcmp(name, "decode_staging")) {
+        if (value < 0 || value > 2) return EKV_ERR_INVALID_ARG;
+        g_decode_staging = value;
         return EKV_OK;
     }
     if (!strcmp(name, "decode_two_term")) {

@@ -18,6 +18,7 @@ extern void *g_profile_ev[2];           // ekv_set_profile_events: recorded arou
 extern int64_t g_decode_merge_slices;   // option "decode_merge_slices"; 0 = automatic, else 1, 4 or 8
 extern int64_t g_attn_out_f32;          // option "attn_out_f32"; 1 = attention entry points store fp32 outputs (debug)
 extern int64_t g_prefill_p_terms;       // option "prefill_p_terms"; 0 = automatic, 1 = one 16-bit term, 2 = two
+extern int64_t g_decode_staging;        // option "decode_staging"; 0 / 1 = cp.async ring (default), 2 = TMA tensor copies (head_dim 128)
 extern int64_t g_decode_two_term;       // option "decode_two_term"; 0 = by the mass test (default), 1 = never, 2 = every step
 extern int64_t g_decode_variant;        // option "decode_variant"; 0 / 3 = ring-staged kernel, 1 = page-stepped comparator
 int decode_chunk_tokens(int batch, int num_kv_heads, int max_seq_len);

@@ -23,6 +23,7 @@
 // decode_page_kernel: the simpler register-direct, page-stepped kernel (no staging, every step is
 // one 16-token page), kept as the plain paged-decode comparator.
 #include "ekv_common.cuh"
+#include <cuda.h>
 #include <math.h>
 #include <string.h>
 #include <atomic>
@@ -539,6 +540,38 @@ struct Step {
 //             Output dim of accumulator (m-tile mt, row g / g+8) is 16 mt + g / 16 mt + 8 + g.
 template <int STAGES> struct RingCfg { static constexpr int kStages = STAGES; };
 
+// Tensor maps of the TMA-staged instantiation (head_dim 128): one layer of a pool seen as
+//   kv_target : [blocks * kv heads * 16 token rows][128 16-bit words], box 64 words x 16 rows, 128-byte swizzle
+//               (K and V; a TARGET slab = two boxes, one per half of the head dimension)
+//   k_base    : [blocks * kv heads * 32 token rows][128 bytes], box 64 bytes x 32 rows, no swizzle
+//               (a BASE K slab = two boxes; rows of 64 bytes alternate between the two halves of the banks)
+//   v_base    : the same bytes, box 128 bytes x 32 rows, 128-byte swizzle (the layout ldmatrix wants)
+struct DecodeMaps {
+    alignas(64) CUtensorMap k_target, v_target, k_base, v_base;
+};
+
+__device__ int g_decode_ring_status = 0;           // 0 ok; 1 = a bounded wait for a staged slab expired (results invalid)
+constexpr int kRingSpinLimit = 1 << 24;
+
+__device__ __forceinline__ void ring_tma_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 :: "r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+// Bounded wait for a phase of an mbarrier; false when the limit is hit.
+__device__ __forceinline__ bool ring_mbar_wait(uint32_t bar, uint32_t parity)
+{
+    for (int i = 0; i < kRingSpinLimit; ++i) {
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\t"
+                     "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                     "selp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+
 __device__ __forceinline__ void ring_cp16(uint32_t dst, const void *src)
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(dst), "l"(src) : "memory");
@@ -560,9 +593,10 @@ __device__ __forceinline__ void ldsm_b8_x2_trans(uint32_t addr, uint32_t &r0, ui
                  : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
 }
 
-template <int D, bool HAS_BASE, int STAGES, int MIN_CTAS, bool BOUNDS = false, bool F16 = false>
-__global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(DecodeParams p)
+template <int D, bool HAS_BASE, int STAGES, int MIN_CTAS, bool BOUNDS = false, bool F16 = false, bool TMA = false>
+__global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(DecodeParams p, const __grid_constant__ DecodeMaps maps)
 {
+    static_assert(!TMA || D == 128, "the TMA-staged instantiation is for head_dim 128");
     static_assert(D == 128 || D == 64, "head_dim");
     constexpr int KS = D / 16;
     constexpr int MT = D / 16;
@@ -570,7 +604,7 @@ __global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(D
     constexpr int kSlot = 2 * kSlab;      // K slab + V slab
     constexpr int CPR_T = D / 8;          // 16-byte chunks per TARGET row
     constexpr int CPR_B = D / 16;         // per BASE row
-    extern __shared__ __align__(128) uint8_t dsm[];
+    extern __shared__ __align__(1024) uint8_t dsm[];
     // Launched with programmatic stream serialisation: nothing in global memory is touched before
     // the previous kernel of the stream (a transition commit, the caller's producer of q) is done.
     cudaGridDependencySynchronize();
@@ -579,6 +613,8 @@ __global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(D
     float (*sm_m)[8] = (float (*)[8])((uint8_t *)sm_q + KS * 32 * sizeof(uint2));
     float (*sm_l)[8] = sm_m + kDecodeWarps;
     uint2 *sm_steps = (uint2 *)(sm_l + kDecodeWarps);     // [4 warps][64] step descriptors
+    // after them: the parked scores (kDecodeThreads x 32 bytes), then, for the TMA-staged instantiation, the
+    // "slab landed" mbarriers [4 warps][K: STAGES, V: STAGES]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int c = lane >> 2, j = lane & 3;
@@ -666,12 +702,49 @@ __global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(D
 
     const uint32_t ring0 = (uint32_t)__cvta_generic_to_shared(dsm) + warp * (STAGES * kSlot);
     const int64_t head_off = (int64_t)g * kSlab;
+    const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(sm_steps + kDecodeWarps * 64) + kDecodeThreads * 32 + warp * (2 * STAGES * 8);
+    bool dead = false;                                     // a bounded wait expired: stop waiting, report
+    if (TMA) {
+        if (lane == 0) {
+#pragma unroll
+            for (int i = 0; i < 2 * STAGES; ++i)
+                asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar0 + 8 * i), "r"(1) : "memory");
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        __syncwarp();
+    }
+    // wait until the K (which = 0) or V (which = 1) slab of step k has landed in its slot
+    auto landed = [&](int k, int slot, int which) {
+        if (TMA) {
+            if (!dead && !ring_mbar_wait(bar0 + 8 * (which * STAGES + slot), (uint32_t)((k / STAGES) & 1))) dead = true;
+        } else {
+            asm volatile("cp.async.wait_group %0;" :: "n"(2 * STAGES - 1) : "memory");
+        }
+        __syncwarp();
+    };
 
     // producer: copy the K and V slabs of a step into ring slot `slot` (8 + 8 x 16 B per lane at D = 128)
     // producer: copy the K (which = 0) or V (which = 1) slab of a step into ring slot `slot`
     auto issue = [&](const Step &st, int slot, int which) {
-        const uint8_t *src = (which ? p.v_layer : p.k_layer) + (int64_t)st.phys * p.block_bytes + head_off;
         const uint32_t dst = ring0 + slot * kSlot + which * kSlab;
+        if (TMA) {
+            // one lane posts the byte count and issues the tensor copies of the slab (two boxes, or one for a BASE V slab)
+            if (lane == 0) {
+                const uint32_t bar = bar0 + 8 * (which * STAGES + slot);
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(kSlab) : "memory");
+                const int slab = st.phys * p.num_kv_heads + g;
+                if (HAS_BASE && st.base) {
+                    if (which) ring_tma_2d(dst, &maps.v_base, 0, slab * 32, bar);
+                    else { ring_tma_2d(dst, &maps.k_base, 0, slab * 32, bar); ring_tma_2d(dst + kSlab / 2, &maps.k_base, 64, slab * 32, bar); }
+                } else {
+                    const CUtensorMap *m = which ? &maps.v_target : &maps.k_target;
+                    ring_tma_2d(dst, m, 0, slab * 16, bar);
+                    ring_tma_2d(dst + kSlab / 2, m, 64, slab * 16, bar);
+                }
+            }
+            return;
+        }
+        const uint8_t *src = (which ? p.v_layer : p.k_layer) + (int64_t)st.phys * p.block_bytes + head_off;
         if (HAS_BASE && st.base) {
 #pragma unroll
             for (int q = 0; q < kSlab / 512; ++q) {
@@ -690,7 +763,7 @@ __global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(D
             }
         }
     };
-    auto commit = [&]() { asm volatile("cp.async.commit_group;" ::: "memory"); };
+    auto commit = [&]() { if (!TMA) asm volatile("cp.async.commit_group;" ::: "memory"); };
     auto rescale = [&](const float (&alpha)[2]) {            // O^T accumulators: columns = heads 2j, 2j + 1
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) { o[mt][0] *= alpha[0]; o[mt][1] *= alpha[1]; o[mt][2] *= alpha[0]; o[mt][3] *= alpha[1]; }
@@ -723,8 +796,7 @@ __global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(D
     for (int k = 0; k < n_steps; ++k) {
         const Step cur = step_at(k);
         const int valid = (t1 - t0) - cur.tok0;
-        asm volatile("cp.async.wait_group %0;" :: "n"(2 * STAGES - 1) : "memory");      // K of this step landed
-        __syncwarp();
+        landed(k, slot, 0);                                     // K of this step landed
         const uint32_t kslot = ring0 + slot * kSlot, vslot = kslot + kSlab;
         const bool more = k + STAGES < n_steps;
         Step nxt{0, 0, 0};
@@ -747,7 +819,8 @@ __global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(D
                     for (int nt = 0; nt < 4; ++nt) {
                         // row c / c + 8 of m-tile nt / 2 is token 16 (nt / 2) + 4 (c / 2) + c % 2 (+ 2 for the upper rows)
                         const int row = 16 * (nt >> 1) + 4 * (c >> 1) + 2 * (nt & 1) + (c & 1);
-                        lds16B(kslot + row * (CPR_B * 16) + (((j + (CPR_B / 2) * a) ^ ((row & 1) * (CPR_B / 2))) << 4), x[nt]);
+                        if (TMA) lds16B(kslot + a * (kSlab / 2) + row * 64 + (j << 4), x[nt]);     // [half of the head dimension][token][64 bytes]
+                        else lds16B(kslot + row * (CPR_B * 16) + (((j + (CPR_B / 2) * a) ^ ((row & 1) * (CPR_B / 2))) << 4), x[nt]);
                     }
 #pragma unroll
                     for (int w = 0; w < 4; ++w) {
@@ -773,8 +846,7 @@ __global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(D
             float alpha[2];
             bool two_term;
             softmax_step_t<2, true, F16>(s, valid, c, m_run, l_run, pb, alpha, thr_abs, two_term, save_addr);
-            asm volatile("cp.async.wait_group %0;" :: "n"(2 * STAGES - 1) : "memory");  // V of this step landed
-            __syncwarp();
+            landed(k, slot, 1);                                 // V of this step landed
             if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) rescale(alpha);      // the running maxima rarely move
             // V: 16 tokens x 16 dims per 8-bit transposing ldmatrix: r0 = tokens 4j..4j+3 of dim c,
             // r1 = the same tokens of dim c + 8; two matrices (two m-tiles) per instruction
@@ -827,7 +899,8 @@ __global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(D
 #pragma unroll
                     for (int nt = 0; nt < 2; ++nt) {           // rows c and c + 8 of the m-tile
                         const int row = nt * 8 + c;
-                        lds16B(kslot + row * (CPR_T * 16) + ((lch ^ (row & 1)) << 4), x[nt]);
+                        if (TMA) lds16B(kslot + (lch >> 3) * (kSlab / 2) + row * 128 + (((lch & 7) ^ (row & 7)) << 4), x[nt]);   // [half][token][128 bytes], hardware swizzle
+                        else lds16B(kslot + row * (CPR_T * 16) + ((lch ^ (row & 1)) << 4), x[nt]);
                     }
                     const uint2 q0 = sm_q[2 * cc][lane], q1 = sm_q[2 * cc + 1][lane];
                     mma_16816<F16>(acc[0][0], acc[0][1], acc[0][2], acc[0][3], x[0][0], x[1][0], x[0][1], x[1][1], q0.x, q0.y,
@@ -845,8 +918,7 @@ __global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(D
             float alpha[2];
             bool two_term;
             softmax_step_t<1, false, F16>(s, valid, c, m_run, l_run, pb, alpha, thr_abs, two_term, save_addr);
-            asm volatile("cp.async.wait_group %0;" :: "n"(2 * STAGES - 1) : "memory");
-            __syncwarp();
+            landed(k, slot, 1);
             if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) rescale(alpha);
             // V: ldmatrix.x4.trans delivers the V^T A-fragments of one m-tile (16 dims x 16 tokens)
             auto pv_target = [&](const uint32_t (&pf)[2]) {
@@ -856,12 +928,13 @@ __global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(D
                     mhi = (2 * j + 8 < valid ? 0x0000ffffu : 0u) | (2 * j + 9 < valid ? 0xffff0000u : 0u);
                 }
                 const int vrow = (lane & 7) + 8 * (lane >> 4);
-                const uint32_t rowp = vslot + vrow * (CPR_T * 16);
+                const uint32_t rowp = vslot + vrow * (TMA ? 128 : CPR_T * 16);
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt) {
                     const int ch = 2 * mt + ((lane >> 3) & 1);
                     uint32_t a0, a1, a2, a3;
-                    ldsm_x4_trans(rowp + (((ch ^ (vrow & 7)) & (CPR_T - 1)) << 4), a0, a1, a2, a3);
+                    if (TMA) ldsm_x4_trans(rowp + (ch >> 3) * (kSlab / 2) + (((ch & 7) ^ (vrow & 7)) << 4), a0, a1, a2, a3);
+                    else ldsm_x4_trans(rowp + (((ch ^ (vrow & 7)) & (CPR_T - 1)) << 4), a0, a1, a2, a3);
                     mma_16816<F16>(o[mt][0], o[mt][1], o[mt][2], o[mt][3], a0 & mlo, a1 & mlo, a2 & mhi, a3 & mhi,
                               pf[0], pf[1], o[mt][0], o[mt][1], o[mt][2], o[mt][3]);
                 }
@@ -890,6 +963,7 @@ __global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(D
         }
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
+    if (TMA && dead) atomicExch(&g_decode_ring_status, 1);
 
     // ---- merge the warps of this CTA (the ring is dead: reuse it for the partial outputs) ----
     __syncthreads();
@@ -950,7 +1024,7 @@ template <int D, int STAGES>
 constexpr size_t ring_smem_bytes()
 {
     return (size_t)kDecodeWarps * STAGES * (2 * kPageSize * D * 2) + (D / 16) * 32 * sizeof(uint2)
-           + 2 * kDecodeWarps * 8 * sizeof(float) + kDecodeWarps * 64 * sizeof(uint2) + kDecodeThreads * 32;
+           + 2 * kDecodeWarps * 8 * sizeof(float) + kDecodeWarps * 64 * sizeof(uint2) + kDecodeThreads * 32 + kDecodeWarps * 2 * STAGES * 8;
 }
 
 // Combine the per-split partials of one (request, query head) row: weights 2^(lse_s - max).
@@ -1099,6 +1173,65 @@ size_t decode_workspace_bytes(int batch, int num_q_heads, int num_kv_heads, int 
 
 using namespace ekv;
 
+// ---- tensor maps of the TMA-staged decode kernel (host) ----
+namespace ekv {
+
+static int encode_2d(CUtensorMap *map, CUtensorMapDataType type, int elem_bytes, const void *base, uint64_t rows,
+                     uint32_t box_x, uint32_t box_rows, CUtensorMapSwizzle swizzle)
+{
+    typedef CUresult (*encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static encode_fn encode = [] {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) fn = nullptr;
+        return (encode_fn)fn;
+    }();
+    if (!encode) return EKV_ERR_CUDA;
+    // a row is 128 elements: 256 bytes of 16-bit words (16 rows per slab) or 128 bytes (32 rows per slab)
+    const cuuint64_t dims1[2] = {(cuuint64_t)128, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)(128 * elem_bytes)};
+    const cuuint32_t box[2] = {box_x, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult rc = encode(map, type, 2, const_cast<void *>(base), dims1, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                               swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return rc == CUDA_SUCCESS ? EKV_OK : EKV_ERR_CUDA;
+}
+
+// The four maps of one (device, layer base pair, pool geometry); the last few are kept, since a serving loop
+// calls with the same pool over and over and an encode costs about a microsecond of host time each.
+static int decode_maps_for(const uint8_t *k_layer, const uint8_t *v_layer, int num_blocks, int num_kv_heads, bool need_base, DecodeMaps *out)
+{
+    struct Entry { const uint8_t *k, *v; int nb, hkv, dev; bool base; DecodeMaps maps; };
+    constexpr int kKeep = 8;
+    static thread_local Entry cache[kKeep];
+    static thread_local int next = 0, used = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return EKV_ERR_CUDA;
+    for (int i = 0; i < used; ++i) {
+        const Entry &e = cache[i];
+        if (e.k == k_layer && e.v == v_layer && e.nb == num_blocks && e.hkv == num_kv_heads && e.dev == dev && (e.base || !need_base)) {
+            *out = e.maps;
+            return EKV_OK;
+        }
+    }
+    Entry &e = cache[next];
+    const uint64_t rows16 = (uint64_t)num_blocks * num_kv_heads * kPageSize;     // TARGET view: 16 rows of 128 words per slab
+    int rc = encode_2d(&e.maps.k_target, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, k_layer, rows16, 64, 16, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (!rc) rc = encode_2d(&e.maps.v_target, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, v_layer, rows16, 64, 16, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (!rc) rc = encode_2d(&e.maps.k_base, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, k_layer, 2 * rows16, 64, 32, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (!rc) rc = encode_2d(&e.maps.v_base, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, v_layer, 2 * rows16, 128, 32, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc) return rc;
+    e.k = k_layer; e.v = v_layer; e.nb = num_blocks; e.hkv = num_kv_heads; e.dev = dev; e.base = true;
+    *out = e.maps;
+    next = (next + 1) % kKeep;
+    if (used < kKeep) ++used;
+    return EKV_OK;
+}
+
+} // namespace ekv
+
 static int decode_impl(const ekv_pool *pool, int32_t layer, const ekv_batch *batch, const int32_t *boundaries,
                        const void *q, void *out, int32_t num_q_heads, float sm_scale,
                        int32_t max_seq_len, void *workspace, size_t workspace_bytes, void *stream)
@@ -1155,12 +1288,26 @@ static int decode_impl(const ekv_pool *pool, int32_t layer, const ekv_batch *bat
     if (f16 && variant == 1) return EKV_ERR_UNSUPPORTED;      // the comparator kernel is bf16 only
     const unsigned nb = (unsigned)ctas;
     cudaError_t aerr = cudaSuccess;
-#define EKV_LAUNCH_RING_T(DD, HB, BD, FF)                                                                 \
+    // Staging of the K/V slabs: cp.async (16 bytes per lane and instruction) by default; with "decode_staging" = 2,
+    // at head_dim 128, tensor copies (TMA: one lane issues two box copies per slab, completion on an mbarrier).
+    // Measured 1-2 % slower than cp.async on every decode configuration, so it is kept as an option only.
+    const bool tma = pool->head_dim == 128 && variant != 1 && g_decode_staging == 2;
+    DecodeMaps maps{};
+    if (tma) {
+        if ((int64_t)pool->num_blocks * pool->num_kv_heads * 32 > 0x7fffffffLL) return EKV_ERR_UNSUPPORTED;    // row coordinates are 32-bit
+        const int mrc = decode_maps_for(p.k_layer, p.v_layer, pool->num_blocks, pool->num_kv_heads, hb, &maps);
+        if (mrc) return mrc;
+    }
+#define EKV_LAUNCH_RING_M(DD, HB, BD, FF, TT)                                                             \
     do {                                                                                                  \
-        aerr = cudaFuncSetAttribute(decode_ring_kernel<DD, HB, 2, 3, BD, FF>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+        aerr = cudaFuncSetAttribute(decode_ring_kernel<DD, HB, 2, 3, BD, FF, TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                     (int)ring_smem_bytes<DD, 2>());                                       \
         if (aerr == cudaSuccess)                                                                          \
-            aerr = launch_pdl(decode_ring_kernel<DD, HB, 2, 3, BD, FF>, nb, kDecodeThreads, ring_smem_bytes<DD, 2>(), st, p); \
+            aerr = launch_pdl(decode_ring_kernel<DD, HB, 2, 3, BD, FF, TT>, nb, kDecodeThreads, ring_smem_bytes<DD, 2>(), st, p, maps); \
+    } while (0)
+#define EKV_LAUNCH_RING_T(DD, HB, BD, FF)                                                                 \
+    do {                                                                                                  \
+        if (DD == 128 && tma) EKV_LAUNCH_RING_M(128, HB, BD, FF, true); else EKV_LAUNCH_RING_M(DD, HB, BD, FF, false); \
     } while (0)
 #define EKV_LAUNCH_RING_B(DD, HB, BD)                                                                     \
     do {                                                                                                  \
@@ -1188,6 +1335,7 @@ static int decode_impl(const ekv_pool *pool, int32_t layer, const ekv_batch *bat
 #undef EKV_LAUNCH_RING
 #undef EKV_LAUNCH_RING_B
 #undef EKV_LAUNCH_RING_T
+#undef EKV_LAUNCH_RING_M
     if (aerr != cudaSuccess) return EKV_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? EKV_OK : EKV_ERR_CUDA;
 }
@@ -1313,4 +1461,14 @@ extern "C" int ekv_attn_decode_noalloc(const ekv_pool *pool, int32_t layer, cons
     // so nothing in the array has to start at zero and nothing is cleared.
     return ekv_attn_decode(pool, layer, batch, q, out, num_q_heads, sm_scale, max_seq_len,
                            scratch, ekv::kNoAllocScratchBytes, stream);
+}
+
+// Host-synchronising debug query: status word of the TMA-staged decode kernel since the last call. Resets the word.
+extern "C" int ekv_decode_status(void)
+{
+    int v = -1, zero = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess) return EKV_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(&v, ekv::g_decode_ring_status, sizeof(int)) != cudaSuccess) return EKV_ERR_CUDA;
+    if (cudaMemcpyToSymbol(ekv::g_decode_ring_status, &zero, sizeof(int)) != cudaSuccess) return EKV_ERR_CUDA;
+    return v;
 }

@@ -179,3 +179,23 @@ def test_growing_scores_across_splits(oracle):
     wl.q[:, :, 0] = synth.f32_to_bf16_bits(np.full(wl.q.shape[:2], 4.0, np.float32))
     for chunk in (0, 256):
         _check(oracle, wl, chunk, what=f"growing scores chunk{chunk}")
+
+
+@pytest.mark.parametrize("frac", [0.0, 0.5, 1.0])
+def test_tma_staging_matches_cp_async(oracle, frac):
+    """Option decode_staging = 2 (tensor copies into the ring, head_dim 128) changes how the slabs travel,
+    not what is computed: outputs equal the default path's bit for bit, and no bounded wait expires."""
+    b = require_gpu()
+    wl = synth.make_workload("tma", seed=808, seq_lens=[1500, 257, 64, 33, 1, 900], num_q_heads=8, num_kv_heads=2, head_dim=128,
+                             base_fraction=frac)
+    op, *_ = mixed_oracle_pool(oracle, wl)
+    pool, batch, q = upload_state(b, op, wl.q)
+    ref = gpu_decode(b, pool, batch, q, wl.num_q_heads, wl.sm_scale)
+    b.ekv_set_option("decode_staging", 2)
+    try:
+        got = gpu_decode(b, pool, batch, q, wl.num_q_heads, wl.sm_scale)
+    finally:
+        b.ekv_set_option("decode_staging", 0)
+    assert b.ekv_decode_status() == 0
+    assert np.array_equal(got, ref)
+    assert_attn_close(got, oracle.attn_decode(op, 0, wl.q, wl.num_q_heads, wl.sm_scale), f"tma f={frac}")
