@@ -791,165 +791,147 @@ __global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(D
     }
     __syncthreads();
 
-    int slot = 0;
-#pragma unroll 1
-    for (int k = 0; k < n_steps; ++k) {
-        const Step cur = step_at(k);
-        const int valid = (t1 - t0) - cur.tok0;
-        landed(k, slot, 0);                                     // K of this step landed
-        const uint32_t kslot = ring0 + slot * kSlot, vslot = kslot + kSlab;
-        const bool more = k + STAGES < n_steps;
-        Step nxt{0, 0, 0};
-        if (more) nxt = step_at(k + STAGES);
-
-        if (HAS_BASE && cur.base) {
-            // S^T = K Q^T: two m-tiles of 16 tokens, heads on the N axis; the K bytes become the A operand
-            // (rows c and c + 8 of m-tile mt are the slab rows that the loop below calls nt = 2 mt, 2 mt + 1)
-            float s[2][4];
-            {
-                float acc[2][2][4];                            // [m-tile][half of the head dimension]: four independent chains
+    // ---- the parts of a step ----
+    // S^T = K Q^T of a BASE step: two m-tiles of 16 tokens, heads on the N axis; the K bytes become the A operand
+    // (rows c and c + 8 of m-tile mt are the slab rows that the loop below calls nt = 2 mt, 2 mt + 1)
+    auto qk_base = [&](uint32_t kslot, float (&s)[2][4]) {
+        float acc[2][2][4];                                    // [m-tile][half of the head dimension]: four independent chains
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int a = 0; a < 2; ++a) acc[mt][a][0] = acc[mt][a][1] = acc[mt][a][2] = acc[mt][a][3] = 0.f;
+#pragma unroll
+        for (int a = 0; a < (KS + 3) / 4; ++a) {               // one 16-byte chunk = 4 k-steps
+            uint32_t x[4][4];
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                // row c / c + 8 of m-tile nt / 2 is token 16 (nt / 2) + 4 (c / 2) + c % 2 (+ 2 for the upper rows)
+                const int row = 16 * (nt >> 1) + 4 * (c >> 1) + 2 * (nt & 1) + (c & 1);
+                if (TMA) lds16B(kslot + a * (kSlab / 2) + row * 64 + (j << 4), x[nt]);     // [half of the head dimension][token][64 bytes]
+                else lds16B(kslot + row * (CPR_B * 16) + (((j + (CPR_B / 2) * a) ^ ((row & 1) * (CPR_B / 2))) << 4), x[nt]);
+            }
+#pragma unroll
+            for (int w = 0; w < 4; ++w) {
+                const uint2 qf = sm_q[4 * a + w][lane];
 #pragma unroll
                 for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-                    for (int a = 0; a < 2; ++a) acc[mt][a][0] = acc[mt][a][1] = acc[mt][a][2] = acc[mt][a][3] = 0.f;
-#pragma unroll
-                for (int a = 0; a < (KS + 3) / 4; ++a) {       // one 16-byte chunk = 4 k-steps
-                    uint32_t x[4][4];
-#pragma unroll
-                    for (int nt = 0; nt < 4; ++nt) {
-                        // row c / c + 8 of m-tile nt / 2 is token 16 (nt / 2) + 4 (c / 2) + c % 2 (+ 2 for the upper rows)
-                        const int row = 16 * (nt >> 1) + 4 * (c >> 1) + 2 * (nt & 1) + (c & 1);
-                        if (TMA) lds16B(kslot + a * (kSlab / 2) + row * 64 + (j << 4), x[nt]);     // [half of the head dimension][token][64 bytes]
-                        else lds16B(kslot + row * (CPR_B * 16) + (((j + (CPR_B / 2) * a) ^ ((row & 1) * (CPR_B / 2))) << 4), x[nt]);
-                    }
-#pragma unroll
-                    for (int w = 0; w < 4; ++w) {
-                        const uint2 qf = sm_q[4 * a + w][lane];
-#pragma unroll
-                        for (int mt = 0; mt < 2; ++mt)
-                            mma_16816<F16>(acc[mt][a & 1][0], acc[mt][a & 1][1], acc[mt][a & 1][2], acc[mt][a & 1][3],
-                                      prmt(x[2 * mt][w], 0u, 0x1404), prmt(x[2 * mt + 1][w], 0u, 0x1404),
-                                      prmt(x[2 * mt][w], 0u, 0x3424), prmt(x[2 * mt + 1][w], 0u, 0x3424),
-                                      qf.x, qf.y,
-                                      acc[mt][a & 1][0], acc[mt][a & 1][1], acc[mt][a & 1][2], acc[mt][a & 1][3]);
-                    }
-                }
-#pragma unroll
-                for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) s[mt][i] = (acc[mt][0][i] + acc[mt][1][i]) * p.scale_log2;
-            }
-            __syncwarp();                                      // every lane has read this K slab: refill it
-            if (more) issue(nxt, slot, 0);
-            commit();
-            uint32_t pb[4];
-            float alpha[2];
-            bool two_term;
-            softmax_step_t<2, true, F16>(s, valid, c, m_run, l_run, pb, alpha, thr_abs, two_term, save_addr);
-            landed(k, slot, 1);                                 // V of this step landed
-            if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) rescale(alpha);      // the running maxima rarely move
-            // V: 16 tokens x 16 dims per 8-bit transposing ldmatrix: r0 = tokens 4j..4j+3 of dim c,
-            // r1 = the same tokens of dim c + 8; two matrices (two m-tiles) per instruction
-            auto pv_base = [&](const uint32_t (&pf)[4]) {
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    // 0 * NaN must not leak from rows past the end: a token byte past the end is replaced by
-                    // the zero byte of the permute's second operand (selector nibble 4)
-                    uint32_t sel_lo = 0x1404u, sel_hi = 0x3424u;   // bytes (0, 1) / (2, 3) become high halves
-                    if (valid < 32) {
-                        const int rem = valid - (16 * hf + 4 * j);
-                        if (rem < 1) sel_lo = (sel_lo & 0xff0fu) | 0x0040u;      // token 4j
-                        if (rem < 2) sel_lo = (sel_lo & 0x0fffu) | 0x4000u;      // token 4j + 1
-                        if (rem < 3) sel_hi = (sel_hi & 0xff0fu) | 0x0040u;      // token 4j + 2
-                        if (rem < 4) sel_hi = (sel_hi & 0x0fffu) | 0x4000u;      // token 4j + 3
-                    }
-                    const int vrow = 16 * hf + (lane & 15);
-                    const uint32_t rowp = vslot + vrow * (CPR_B * 16);
-#pragma unroll
-                    for (int mp = 0; mp < MT / 2; ++mp) {
-                        const int ch = 2 * mp + (lane >> 4);
-                        uint32_t r0, r1, r2, r3;
-                        ldsm_b8_x2_trans(rowp + (((ch ^ (vrow & 7)) & (CPR_B - 1)) << 4), r0, r1, r2, r3);
-                        mma_16816<F16>(o[2 * mp][0], o[2 * mp][1], o[2 * mp][2], o[2 * mp][3],
-                                  prmt(r0, 0u, sel_lo), prmt(r1, 0u, sel_lo), prmt(r0, 0u, sel_hi), prmt(r1, 0u, sel_hi),
-                                  pf[2 * hf], pf[2 * hf + 1], o[2 * mp][0], o[2 * mp][1], o[2 * mp][2], o[2 * mp][3]);
-                        mma_16816<F16>(o[2 * mp + 1][0], o[2 * mp + 1][1], o[2 * mp + 1][2], o[2 * mp + 1][3],
-                                  prmt(r2, 0u, sel_lo), prmt(r3, 0u, sel_lo), prmt(r2, 0u, sel_hi), prmt(r3, 0u, sel_hi),
-                                  pf[2 * hf], pf[2 * hf + 1],
-                                  o[2 * mp + 1][0], o[2 * mp + 1][1], o[2 * mp + 1][2], o[2 * mp + 1][3]);
-                    }
-                }
-            };
-            pv_base(pb);
-            if (two_term) {                                    // rare, uniform over the warp: the low-order terms of P
-                uint32_t pl[4];
-                two_term_residuals<2, F16>(save_addr, m_run, pl);
-                pv_base(pl);
-            }
-        } else {
-            float s[1][4];
-            {
-                float acc[2][4];                               // one m-tile of 16 tokens; two chains over the k-steps
-#pragma unroll
-                for (int a = 0; a < 2; ++a) acc[a][0] = acc[a][1] = acc[a][2] = acc[a][3] = 0.f;
-#pragma unroll
-                for (int cc = 0; cc < KS / 2; ++cc) {          // one 16-byte chunk = 2 k-steps
-                    const int lch = 2 * j + (cc & 1) + (CPR_T / 2) * (cc >> 1);
-                    uint32_t x[2][4];
-#pragma unroll
-                    for (int nt = 0; nt < 2; ++nt) {           // rows c and c + 8 of the m-tile
-                        const int row = nt * 8 + c;
-                        if (TMA) lds16B(kslot + (lch >> 3) * (kSlab / 2) + row * 128 + (((lch & 7) ^ (row & 7)) << 4), x[nt]);   // [half][token][128 bytes], hardware swizzle
-                        else lds16B(kslot + row * (CPR_T * 16) + ((lch ^ (row & 1)) << 4), x[nt]);
-                    }
-                    const uint2 q0 = sm_q[2 * cc][lane], q1 = sm_q[2 * cc + 1][lane];
-                    mma_16816<F16>(acc[0][0], acc[0][1], acc[0][2], acc[0][3], x[0][0], x[1][0], x[0][1], x[1][1], q0.x, q0.y,
-                              acc[0][0], acc[0][1], acc[0][2], acc[0][3]);
-                    mma_16816<F16>(acc[1][0], acc[1][1], acc[1][2], acc[1][3], x[0][2], x[1][2], x[0][3], x[1][3], q1.x, q1.y,
-                              acc[1][0], acc[1][1], acc[1][2], acc[1][3]);
-                }
-#pragma unroll
-                for (int i = 0; i < 4; ++i) s[0][i] = (acc[0][i] + acc[1][i]) * p.scale_log2;
-            }
-            __syncwarp();
-            if (more) issue(nxt, slot, 0);
-            commit();
-            uint32_t pb[2];
-            float alpha[2];
-            bool two_term;
-            softmax_step_t<1, false, F16>(s, valid, c, m_run, l_run, pb, alpha, thr_abs, two_term, save_addr);
-            landed(k, slot, 1);
-            if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) rescale(alpha);
-            // V: ldmatrix.x4.trans delivers the V^T A-fragments of one m-tile (16 dims x 16 tokens)
-            auto pv_target = [&](const uint32_t (&pf)[2]) {
-                uint32_t mlo = 0xffffffffu, mhi = 0xffffffffu;     // tokens 2j, 2j+1 | 2j+8, 2j+9
-                if (valid < kPageSize) {
-                    mlo = (2 * j < valid ? 0x0000ffffu : 0u) | (2 * j + 1 < valid ? 0xffff0000u : 0u);
-                    mhi = (2 * j + 8 < valid ? 0x0000ffffu : 0u) | (2 * j + 9 < valid ? 0xffff0000u : 0u);
-                }
-                const int vrow = (lane & 7) + 8 * (lane >> 4);
-                const uint32_t rowp = vslot + vrow * (TMA ? 128 : CPR_T * 16);
-#pragma unroll
-                for (int mt = 0; mt < MT; ++mt) {
-                    const int ch = 2 * mt + ((lane >> 3) & 1);
-                    uint32_t a0, a1, a2, a3;
-                    if (TMA) ldsm_x4_trans(rowp + (ch >> 3) * (kSlab / 2) + (((ch & 7) ^ (vrow & 7)) << 4), a0, a1, a2, a3);
-                    else ldsm_x4_trans(rowp + (((ch ^ (vrow & 7)) & (CPR_T - 1)) << 4), a0, a1, a2, a3);
-                    mma_16816<F16>(o[mt][0], o[mt][1], o[mt][2], o[mt][3], a0 & mlo, a1 & mlo, a2 & mhi, a3 & mhi,
-                              pf[0], pf[1], o[mt][0], o[mt][1], o[mt][2], o[mt][3]);
-                }
-            };
-            pv_target(pb);
-            if (two_term) {
-                uint32_t pl[2];
-                two_term_residuals<1, F16>(save_addr, m_run, pl);
-                pv_target(pl);
+                    mma_16816<F16>(acc[mt][a & 1][0], acc[mt][a & 1][1], acc[mt][a & 1][2], acc[mt][a & 1][3],
+                              prmt(x[2 * mt][w], 0u, 0x1404), prmt(x[2 * mt + 1][w], 0u, 0x1404),
+                              prmt(x[2 * mt][w], 0u, 0x3424), prmt(x[2 * mt + 1][w], 0u, 0x3424),
+                              qf.x, qf.y,
+                              acc[mt][a & 1][0], acc[mt][a & 1][1], acc[mt][a & 1][2], acc[mt][a & 1][3]);
             }
         }
-        __syncwarp();                                          // every lane is done with this slot
-        if (more) issue(nxt, slot, 1);                        // the V slab of this slot is free now
-        commit();
-        slot = slot + 1 == STAGES ? 0 : slot + 1;
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) s[mt][i] = (acc[mt][0][i] + acc[mt][1][i]) * p.scale_log2;
+    };
+    // S^T of a TARGET step: one m-tile of 16 tokens (in s[0]); two chains over the k-steps
+    auto qk_target = [&](uint32_t kslot, float (&s)[2][4]) {
+        float acc[2][4];
+#pragma unroll
+        for (int a = 0; a < 2; ++a) acc[a][0] = acc[a][1] = acc[a][2] = acc[a][3] = 0.f;
+#pragma unroll
+        for (int cc = 0; cc < KS / 2; ++cc) {                  // one 16-byte chunk = 2 k-steps
+            const int lch = 2 * j + (cc & 1) + (CPR_T / 2) * (cc >> 1);
+            uint32_t x[2][4];
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) {                   // rows c and c + 8 of the m-tile
+                const int row = nt * 8 + c;
+                if (TMA) lds16B(kslot + (lch >> 3) * (kSlab / 2) + row * 128 + (((lch & 7) ^ (row & 7)) << 4), x[nt]);   // [half][token][128 bytes], hardware swizzle
+                else lds16B(kslot + row * (CPR_T * 16) + ((lch ^ (row & 1)) << 4), x[nt]);
+            }
+            const uint2 q0 = sm_q[2 * cc][lane], q1 = sm_q[2 * cc + 1][lane];
+            mma_16816<F16>(acc[0][0], acc[0][1], acc[0][2], acc[0][3], x[0][0], x[1][0], x[0][1], x[1][1], q0.x, q0.y,
+                      acc[0][0], acc[0][1], acc[0][2], acc[0][3]);
+            mma_16816<F16>(acc[1][0], acc[1][1], acc[1][2], acc[1][3], x[0][2], x[1][2], x[0][3], x[1][3], q1.x, q1.y,
+                      acc[1][0], acc[1][1], acc[1][2], acc[1][3]);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) s[0][i] = (acc[0][i] + acc[1][i]) * p.scale_log2;
+    };
+    // softmax and PV of a BASE step. V: 16 tokens x 16 dims per 8-bit transposing ldmatrix: r0 = tokens 4j..4j+3 of
+    // dim c, r1 = the same tokens of dim c + 8; two matrices (two m-tiles) per instruction
+    auto tail_base = [&](float (&s)[2][4], int valid, uint32_t vslot, int k, int slot) {
+        uint32_t pb[4];
+        float alpha[2];
+        bool two_term;
+        softmax_step_t<2, true, F16>(s, valid, c, m_run, l_run, pb, alpha, thr_abs, two_term, save_addr);
+        landed(k, slot, 1);                                     // V of this step landed
+        if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) rescale(alpha);      // the running maxima rarely move
+        auto pv_base = [&](const uint32_t (&pf)[4]) {
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                // 0 * NaN must not leak from rows past the end: a token byte past the end is replaced by
+                // the zero byte of the permute's second operand (selector nibble 4)
+                uint32_t sel_lo = 0x1404u, sel_hi = 0x3424u;   // bytes (0, 1) / (2, 3) become high halves
+                if (valid < 32) {
+                    const int rem = valid - (16 * hf + 4 * j);
+                    if (rem < 1) sel_lo = (sel_lo & 0xff0fu) | 0x0040u;      // token 4j
+                    if (rem < 2) sel_lo = (sel_lo & 0x0fffu) | 0x4000u;      // token 4j + 1
+                    if (rem < 3) sel_hi = (sel_hi & 0xff0fu) | 0x0040u;      // token 4j + 2
+                    if (rem < 4) sel_hi = (sel_hi & 0x0fffu) | 0x4000u;      // token 4j + 3
+                }
+                const int vrow = 16 * hf + (lane & 15);
+                const uint32_t rowp = vslot + vrow * (CPR_B * 16);
+#pragma unroll
+                for (int mp = 0; mp < MT / 2; ++mp) {
+                    const int ch = 2 * mp + (lane >> 4);
+                    uint32_t r0, r1, r2, r3;
+                    ldsm_b8_x2_trans(rowp + (((ch ^ (vrow & 7)) & (CPR_B - 1)) << 4), r0, r1, r2, r3);
+                    mma_16816<F16>(o[2 * mp][0], o[2 * mp][1], o[2 * mp][2], o[2 * mp][3],
+                              prmt(r0, 0u, sel_lo), prmt(r1, 0u, sel_lo), prmt(r0, 0u, sel_hi), prmt(r1, 0u, sel_hi),
+                              pf[2 * hf], pf[2 * hf + 1], o[2 * mp][0], o[2 * mp][1], o[2 * mp][2], o[2 * mp][3]);
+                    mma_16816<F16>(o[2 * mp + 1][0], o[2 * mp + 1][1], o[2 * mp + 1][2], o[2 * mp + 1][3],
+                              prmt(r2, 0u, sel_lo), prmt(r3, 0u, sel_lo), prmt(r2, 0u, sel_hi), prmt(r3, 0u, sel_hi),
+                              pf[2 * hf], pf[2 * hf + 1],
+                              o[2 * mp + 1][0], o[2 * mp + 1][1], o[2 * mp + 1][2], o[2 * mp + 1][3]);
+                }
+            }
+        };
+        pv_base(pb);
+        if (two_term) {                                        // rare, uniform over the warp: the low-order terms of P
+            uint32_t pl[4];
+            two_term_residuals<2, F16>(save_addr, m_run, pl);
+            pv_base(pl);
+        }
+    };
+    // softmax and PV of a TARGET step. V: ldmatrix.x4.trans delivers the V^T A-fragments of one m-tile (16 dims x 16 tokens)
+    auto tail_target = [&](float (&s2)[2][4], int valid, uint32_t vslot, int k, int slot) {
+        float (&s)[1][4] = *(float (*)[1][4])&s2[0];
+        uint32_t pb[2];
+        float alpha[2];
+        bool two_term;
+        softmax_step_t<1, false, F16>(s, valid, c, m_run, l_run, pb, alpha, thr_abs, two_term, save_addr);
+        landed(k, slot, 1);
+        if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) rescale(alpha);
+        auto pv_target = [&](const uint32_t (&pf)[2]) {
+            uint32_t mlo = 0xffffffffu, mhi = 0xffffffffu;     // tokens 2j, 2j+1 | 2j+8, 2j+9
+            if (valid < kPageSize) {
+                mlo = (2 * j < valid ? 0x0000ffffu : 0u) | (2 * j + 1 < valid ? 0xffff0000u : 0u);
+                mhi = (2 * j + 8 < valid ? 0x0000ffffu : 0u) | (2 * j + 9 < valid ? 0xffff0000u : 0u);
+            }
+            const int vrow = (lane & 7) + 8 * (lane >> 4);
+            const uint32_t rowp = vslot + vrow * (TMA ? 128 : CPR_T * 16);
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                const int ch = 2 * mt + ((lane >> 3) & 1);
+                uint32_t a0, a1, a2, a3;
+                if (TMA) ldsm_x4_trans(rowp + (ch >> 3) * (kSlab / 2) + (((ch & 7) ^ (vrow & 7)) << 4), a0, a1, a2, a3);
+                else ldsm_x4_trans(rowp + (((ch ^ (vrow & 7)) & (CPR_T - 1)) << 4), a0, a1, a2, a3);
+                mma_16816<F16>(o[mt][0], o[mt][1], o[mt][2], o[mt][3], a0 & mlo, a1 & mlo, a2 & mhi, a3 & mhi,
+                          pf[0], pf[1], o[mt][0], o[mt][1], o[mt][2], o[mt][3]);
+            }
+        };
+        pv_target(pb);
+        if (two_term) {
+            uint32_t pl[2];
+            two_term_residuals<1, F16>(save_addr, m_run, pl);
+            pv_target(pl);
+        }
+    };
+    auto refresh_thresholds = [&](int k) {
         if (p.two_term == 0 && ((k & (k + 1)) == 0 || (k & (kTwoTermRefresh - 1)) == kTwoTermRefresh - 1)) {
             // refresh the two-term thresholds (after steps 0, 1, 3, 7, then every 8th) from the warp-wide sums
             float L0 = l_run[0], L1 = l_run[1];
@@ -961,6 +943,29 @@ __global__ void __launch_bounds__(kDecodeThreads, MIN_CTAS) decode_ring_kernel(D
             thr_abs[0] = m_run[0] + __log2f(L0) + kTwoTermLog2Share;
             thr_abs[1] = m_run[1] + __log2f(L1) + kTwoTermLog2Share;
         }
+    };
+
+    int slot = 0;
+#pragma unroll 1
+    for (int k = 0; k < n_steps; ++k) {
+        const Step cur = step_at(k);
+        const int valid = (t1 - t0) - cur.tok0;
+        landed(k, slot, 0);                                     // K of this step landed
+        const uint32_t kslot = ring0 + slot * kSlot, vslot = kslot + kSlab;
+        const bool more = k + STAGES < n_steps;
+        Step nxt{0, 0, 0};
+        if (more) nxt = step_at(k + STAGES);
+        float s[2][4];
+        if (HAS_BASE && cur.base) qk_base(kslot, s); else qk_target(kslot, s);
+        __syncwarp();                                          // every lane has read this K slab: refill it
+        if (more) issue(nxt, slot, 0);
+        commit();
+        if (HAS_BASE && cur.base) tail_base(s, valid, vslot, k, slot); else tail_target(s, valid, vslot, k, slot);
+        __syncwarp();                                          // every lane is done with this slot
+        if (more) issue(nxt, slot, 1);                        // the V slab of this slot is free now
+        commit();
+        slot = slot + 1 == STAGES ? 0 : slot + 1;
+        refresh_thresholds(k);
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     if (TMA && dead) atomicExch(&g_decode_ring_status, 1);
