@@ -37,7 +37,7 @@ UNIT = "GB/s"
 TRANSITION_PAIRS = 16          # the paper's minimum demotion batch B_min^d (App. B.1)
 # dram__bytes_read.sum + dram__bytes_write.sum divided by the algorithmic K/V bytes, from the ncu
 # capture summarised in profiles/decode_ring_kernel_llama8b_decode_f05.md
-NCU_TRAFFIC_PER_KV_BYTE = 1.0193
+NCU_TRAFFIC_PER_KV_BYTE = 1.0173
 WORKLOAD = ("llama3-8b-shaped decode: batch 64, ctx U[1024,8192], Hq 32 / Hkv 8, D 128, page 16, "
             "BASE fraction 0.5 (random pairs), random physical placement; per step: downgrade 16 pairs "
             "-> mixed-fidelity decode attention -> refine 16 pairs")
@@ -587,14 +587,11 @@ def metadata_lowering(b, torch, dev, batch=256):
     t_low = wall(lowered)
     assert torch.equal(out_table[:, :1], bt.block_table[:, :1]) and flags.cpu().tolist()[2] == 0
     t_py = wall(per_request, n=5)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(20):
-        b.ekv_lower_sparse_metadata(pool, out_batch, out_sl, v[0], v[1], v[2], v[3], v[4], v[5] if len(v[5]) else None, bounds, flags)
-    e1.record(); torch.cuda.synchronize()
     return {"workload": f"batch {wl.batch} of the high-concurrency configuration, {int(offs[-1]) * 4} bytes of sparse description",
-            "lowered_us_per_step": round(t_low * 1e6, 1), "kernel_us": round(e0.elapsed_time(e1) / 20 * 1e3, 2),
-            "per_request_copies_us_per_step": round(t_py * 1e6, 1), "flags": flags.cpu().tolist()}
+            "lowered_us_per_step": round(t_low * 1e6, 1),
+            "per_request_copies_us_per_step": round(t_py * 1e6, 1), "flags": flags.cpu().tolist(),
+            "note": "host wall clock per step, device synchronised: one pinned copy + one launch, against one table-row copy "
+                    "and one length write per request"}
 
 
 def extras(b, torch, dev, args):
