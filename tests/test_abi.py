@@ -82,3 +82,51 @@ def test_workspace_sizing(lib):
     batch = binding.ekv_batch(0x4000, 0x5000, 64, 512, 1, 0)
     assert lib.ekv_attn_decode(C.byref(pool), 0, C.byref(batch), 0x6000, 0x7000, 32, 0.1, 8192, 0x100, n - 1, None) == -3
     lib.ekv_set_option(b"decode_chunk_tokens", 0)
+
+
+def test_argument_checks_of_the_later_entry_points(lib):
+    """Lowering, tag reset, the no-workspace decode and the options: refused on the host, no launch."""
+    pool = binding.ekv_pool(0x1000, 0x2000, 0x3000, 8, 2, 64, 16, 1, 0, 8 * 2 * 16 * 64 * 2)
+    batch = binding.ekv_batch(0x4000, 0x5000, 2, 4, 1, 0)
+    low = lambda n=1, sl=0x10, lens=0x20, bs=0x30, ids=0x40, rs=0x50, bounds=0x60, flags=0x70, row_of=None: \
+        lib.ekv_lower_sparse_metadata(C.byref(pool), C.byref(batch), sl, n, row_of, lens, bs, ids, rs, None, bounds, flags, None)
+    assert low(n=-1) == -1
+    assert low(sl=None) == -1 and low(bounds=None) == -1 and low(flags=None) == -1
+    assert low(lens=None) == -1 and low(bs=None) == -1 and low(ids=None) == -1 and low(rs=None) == -1
+    assert low(n=3) == -1                                        # more requests than table rows, no row_of
+    no_tags = binding.ekv_pool(0x1000, 0x2000, None, 8, 2, 64, 16, 1, 0, 8 * 2 * 16 * 64 * 2)
+    assert lib.ekv_lower_sparse_metadata(C.byref(no_tags), C.byref(batch), 0x10, 1, None, 0x20, 0x30, 0x40, 0x50, None,
+                                         0x60, 0x70, None) == -1
+    assert lib.ekv_reset_tags(C.byref(pool), None, 3, None) == -1
+    assert lib.ekv_reset_tags(C.byref(pool), None, 0, None) == 0
+    assert lib.ekv_reset_tags(C.byref(no_tags), 0x10, 1, None) == -1
+    # the no-workspace decode: argument errors first, then the size of its fixed array
+    assert lib.ekv_attn_decode_noalloc(None, 0, C.byref(batch), 0x6000, 0x7000, 8, 0.125, 64, None) == -1
+    assert lib.ekv_attn_decode_noalloc(C.byref(pool), 0, C.byref(batch), 0x6000, 0x7000, 0, 0.125, 64, None) == -1
+    big = binding.ekv_pool(0x1000, 0x2000, 0x3000, 1 << 20, 8, 128, 16, 1, 0, (1 << 20) * 8 * 16 * 128 * 2)
+    bb = binding.ekv_batch(0x4000, 0x5000, 256, 1 << 14, 1, 0)
+    lib.ekv_set_option(b"decode_chunk_tokens", 64)
+    assert lib.ekv_attn_workspace_bytes(C.byref(big), 256, 64, 1 << 18, 0) > lib.ekv_attn_decode_noalloc_max_bytes()
+    assert lib.ekv_attn_decode_noalloc(C.byref(big), 0, C.byref(bb), 0x6000, 0x7000, 64, 0.1, 1 << 18, None) == -3
+    lib.ekv_set_option(b"decode_chunk_tokens", 0)
+    for name, bad in ((b"decode_two_term", 3), (b"prefill_p_terms", 3), (b"decode_staging", 3), (b"attn_out_f32", 2),
+                      (b"decode_merge_slices", 3), (b"decode_variant", 2), (b"prefill_variant", 2)):
+        assert lib.ekv_set_option(name, bad) == -1, name
+        assert lib.ekv_set_option(name, 0) == 0, name
+
+
+def test_split_size_rule(lib):
+    """The automatic split size, read back through the workspace size (partials = rows x splits x (D + 1) floats):
+    small launches get one balanced wave of at most two CTAs per SM, large ones splits of at most 3200 tokens."""
+    pool = binding.ekv_pool(0x1000, 0x2000, 0x3000, 8, 8, 128, 16, 1, 0, 1 << 30)
+
+    def splits(batch, max_len, hq=32):
+        n = lib.ekv_attn_workspace_bytes(C.byref(pool), batch, hq, max_len, 0)
+        rows = batch * hq
+        return 1 if n == 0 else round(n / (rows * 129 * 4))
+    # without a GPU the SM count falls back to 148
+    assert splits(64, 8192) == 3                                 # 3200-token splits
+    assert splits(8, 8192) == 4                                  # 64 units x 4 = 256 CTAs <= 296
+    assert splits(4, 32768) == 9                                 # 32 units x 9 = 288 CTAs
+    assert splits(1, 8192) == 32                                 # floor of 256 tokens
+    assert splits(256, 16384) == 6                               # capped at 3200 tokens: ceil(16384 / 3200)
