@@ -376,43 +376,6 @@ __global__ void __launch_bounds__(kDecodeThreads, 3) decode_page_kernel(DecodePa
     }
 }
 
-// Online-softmax update for one step of NT n-tiles (8 tokens each). s holds the scaled scores
-// (log2 domain) of head c for tokens nt*8 + 2j + {0,1}; on return pb[nt] holds the bf16x2
-// probabilities in B-fragment order and `alpha` the rescale factor of head c.
-// With QUAD_TOKENS the columns of an n-tile pair stand for tokens in groups of four (the order the
-// 8-bit transposing ldmatrix delivers V in): n-tile nt, column 2j + e is token
-// 16 (nt / 2) + 4j + 2 (nt % 2) + e.
-template <int NT, bool QUAD_TOKENS = false, bool F16 = false>
-__device__ __forceinline__ void softmax_step(float (&s)[NT][2], int valid, int j, float &m_run, float &l_run,
-                                             uint32_t (&pb)[NT], float &alpha)
-{
-    if (valid < NT * 8) {
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const int tok = QUAD_TOKENS ? 16 * (nt >> 1) + 4 * j + 2 * (nt & 1) + e : nt * 8 + 2 * j + e;
-                if (tok >= valid) s[nt][e] = -INFINITY;
-            }
-    }
-    float mx = fmaxf(s[0][0], s[0][1]);
-#pragma unroll
-    for (int nt = 1; nt < NT; ++nt) mx = fmaxf(mx, fmaxf(s[nt][0], s[nt][1]));
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-    const float m_new = fmaxf(m_run, mx);            // finite: the first token of a step always exists
-    alpha = fast_exp2(m_run - m_new);
-    float sum = 0.f;
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-        const float p0 = fast_exp2(s[nt][0] - m_new), p1 = fast_exp2(s[nt][1] - m_new);
-        sum += p0 + p1;
-        pb[nt] = pack_16x2<F16>(p0, p1);
-    }
-    l_run = l_run * alpha + sum;
-    m_run = m_new;
-}
-
 // Online-softmax update for one step of the ring kernel, whose QK product has the TOKENS on the M axis
 // (S^T = K Q^T: 16 tokens x 8 heads per MMA, so the MMA rows are all real work and the query heads sit
 // on the 8-wide N axis). acc[mt] is the accumulator of m-tile mt: {c0, c1} = row g, heads 2t, 2t+1;
