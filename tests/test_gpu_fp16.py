@@ -134,3 +134,24 @@ def test_transitions_bit_exact_on_fp16_pool(oracle):
     b.ekv_refine(pool, batch, dev_i32(wl.base_pair_req), dev_i32(wl.base_pair_idx), dfreed, dkr, dvr, dev_i32(np.arange(n)))
     torch.cuda.synchronize()
     assert np.array_equal(words(pool.k_pool), wl.k_pool) and np.array_equal(words(pool.v_pool), wl.v_pool)
+
+
+def test_prefill_two_terms_forced_on_fp16(oracle):
+    """fp16 pools take one probability term by default; with prefill_p_terms = 2 the residual pass runs for
+    them too and the fp32 result comes within 1e-4 of the oracle (one term: about 1.5e-3)."""
+    from gpu_util import assert_attn_close_f32
+    b = require_gpu()
+    wl = synth.make_workload("pf16two", seed=515, seq_lens=[300, 129, 40], num_q_heads=8, num_kv_heads=2, head_dim=128,
+                             chunk_lens=[300, 60, 40], base_fraction=0.5, elem_type="fp16")
+    op, *_ = mixed_oracle_pool(oracle, wl)
+    exp = oracle.attn_prefill_chunk(op, 0, wl.q_start, wl.q, wl.num_q_heads, wl.sm_scale)
+    pool, batch, q = upload_state(b, op, wl.q)
+    b.ekv_set_option("prefill_p_terms", 2)
+    try:
+        got32 = gpu_prefill(b, pool, batch, q, wl, f32=True)
+        got = gpu_prefill(b, pool, batch, q, wl)
+    finally:
+        b.ekv_set_option("prefill_p_terms", 0)
+    assert np.abs(got32 - exp).max() < 1e-4
+    assert_attn_close_f32(got32, exp, "fp16, two terms")
+    assert_attn_close(got, exp, "fp16, two terms", elem_type="fp16")
