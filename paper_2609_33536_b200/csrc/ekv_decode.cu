@@ -5,23 +5,27 @@
 // shared memory at the end and the CTA writes either the final bf16 rows (single split) or an
 // fp32 partial (normalised O and log2-sum-exp) that decode_merge_kernel combines.
 //
-// Tensor-core mapping (both kernels below):
-//   QK^T : mma.m16n8k16, M = query heads of the group (rows 8..15 are zero padding),
-//          N = 8 tokens, K = 16 dims. A dot product does not care in which order the head
-//          dimension is visited, so each lane owns contiguous runs of dims and the query
-//          fragment is laid out with the same ownership: operands are fetched 16 / 32 bytes at
-//          a time, never element-wise.
-//   PV   : transposed, O^T[d][head] += V^T[d][tok] P^T[tok][head]: M = 16 dims, N = 8 heads,
-//          K = 16 tokens. The QK accumulator layout (head = lane/4, tokens 2j, 2j+1) is exactly
-//          the B-fragment layout needed here, so P never leaves registers; the V^T fragment is
-//          made from two token rows with one byte-permute per register.
+// Tensor-core mapping:
+//   decode_ring_kernel (the product path, native and elastic instantiations)
+//     QK^T : S^T = K Q^T, mma.m16n8k16 with M = 16 tokens, N = 8 query heads of the group (columns
+//            past the group are zero queries), K = 16 dims, so every MMA row is real work. A dot
+//            product does not care in which order the head dimension is visited, so each lane owns
+//            contiguous runs of dims and the query fragments are laid out with the same ownership:
+//            operands are fetched 16 bytes at a time, never element-wise.
+//     PV   : transposed, O^T[d][head] += V^T[d][tok] P^T[tok][head]: M = 16 dims, N = 8 heads,
+//            K = 16 tokens. movmatrix turns the packed halves of an S^T accumulator into the B
+//            fragment of P^T, so P never leaves registers; the V^T fragments come from ldmatrix
+//            (16-bit transposing for TARGET slabs, 8-bit transposing plus one byte-permute per
+//            register for BASE slabs).
+//     K and V slabs are staged global -> shared memory through a per-warp ring, two steps ahead
+//     (cp.async by default, TMA tensor copies as an option).
+//     Probabilities enter PV as one 16-bit term, or as two (rounded value + rounding residual) on
+//     steps that hold a heavy token: see softmax_step_t.
+//   decode_page_kernel: an older design kept for A/B runs (option decode_variant = 1): register-
+//     direct, page-stepped (every step is one 16-token page), query heads on the M axis of QK^T
+//     (rows 8..15 are zero padding), bf16 pools only.
 // BASE blocks: half as many bytes are fetched and expanded byte -> (byte << 8) with byte-permute
 // instructions in registers; nothing is materialised in memory.
-//
-// decode_ring_kernel (the product path, native and elastic instantiations): K and V slabs are
-// staged global -> shared memory with cp.async through a per-warp ring, two steps ahead.
-// decode_page_kernel: the simpler register-direct, page-stepped kernel (no staging, every step is
-// one 16-token page), kept as the plain paged-decode comparator.
 #include "ekv_common.cuh"
 #include <cuda.h>
 #include <math.h>
