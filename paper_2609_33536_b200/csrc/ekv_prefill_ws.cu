@@ -33,7 +33,14 @@
 //     memory), move the references, rescale O in TMEM and redo the tile. Exponentials and the
 //     row sum run on packed f32x2 instructions; the probabilities are written as packed 16-bit
 //     pairs over the scores (P aliases S).
-// TMEM columns: S_0/P_0 [0,128), S_1/P_1 [128,256), O_0 [256,384), O_1 [384,512).
+//   - two-term probabilities (template parameter TWO_TERM; the default for bf16 pools): the softmax
+//     thread also forms the rounding residual of every probability (kept negated, hi - p) and writes
+//     it, as 16-bit pairs, into the upper 64 columns of the row tile's score region; the MMA issuer
+//     follows PV_w(j) with a second pass over the same V tile whose A operand is that region, with
+//     the negate-A bit of the instruction descriptor set. One bf16 term alone leaves up to 5e-3 of
+//     output error on rows that two or three tokens dominate.
+// TMEM columns: S_0/P_0 [0,128) (probabilities in [0,64), their residuals in [64,128)), S_1/P_1
+// [128,256) likewise, O_0 [256,384), O_1 [384,512).
 // Every wait on an mbarrier is bounded; on expiry the thread records a status word, stops
 // waiting (it still arrives where others count on it), and the CTA frees its tensor memory.
 #include "ekv_common.cuh"
