@@ -190,7 +190,7 @@ def run_ours(args):
         b.ekv_attn_decode(pool, 0, batch, q, out, wl.num_q_heads, wl.sm_scale, msl, ws)
         b.ekv_refine(pool, batch, d_req, d_idx, freed, kres, vres, d_slot)
 
-    k0 = pool.k_pool.clone() if rank == 0 else None
+    k0 = pool.k_pool.clone()
     for _ in range(max(args.warmup, 3)):
         step()
     torch.cuda.synchronize()
@@ -234,9 +234,9 @@ def run_ours(args):
     main_ms = float(np.mean([e0.elapsed_time(e1) for e0, e1 in prof]))
 
     result = None
-    if rank == 0:
+    if True:                                                # every rank: the end-to-end leg is measured on all of them
         assert torch.equal(pool.k_pool, k0), "pool state drifted across steps"
-        clocks = sampler.stop()
+        clocks = sampler.stop() if sampler else None
         peak, peak_src = _peaks()
         achieved = kv_bytes / (main_ms * 1e-3) / 1e9
         result = {
@@ -260,7 +260,7 @@ def run_ours(args):
         }
         if args.profile_only:
             result["config"]["note"] = "profiling run: reduced batch, no e2e / cpu_baseline / extras"
-            return result
+            return result if rank == 0 else None
         # ---- end to end: host buffers, H2D of the step's inputs and D2H of its result, every step ----
         # The step's inputs (queries, block table, sequence lengths, the transition batch) sit in ONE pinned
         # host arena and travel in one copy to a device arena the calls read through views; the result comes
@@ -326,8 +326,12 @@ def run_ours(args):
         dt = timed_e2e(graph_step, Ke)
         assert torch.equal(outh.view(torch.int16), out_eager.view(torch.int16)), "graph replay and eager step disagree"
         assert torch.equal(pool.k_pool, k0), "pool state drifted across end-to-end steps"
-        result["e2e"] = {"value": round(step_bytes * world / dt / 1e9, 1), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                         "d2h_bytes_per_step": int(d2h), "ms_per_step": round(dt * 1e3, 5), "steps": Ke,
+        # every rank measured its own replica: the job's time is the slowest rank's, its work the sum
+        dt, e2e_bytes = aggregate_over_ranks(dt * 1e3, float(step_bytes), dev)
+        dt *= 1e-3
+        dt_eager = aggregate_over_ranks(dt_eager * 1e3, 0.0, dev)[0] * 1e-3
+        result["e2e"] = {"value": round(e2e_bytes / dt / 1e9, 1), "unit": UNIT, "h2d_bytes_per_step": h2d * world,
+                         "d2h_bytes_per_step": int(d2h) * world, "ms_per_step": round(dt * 1e3, 5), "steps": Ke,
                          "eager_ms_per_step": round(dt_eager * 1e3, 5),
                          "note": "host wall clock, one stream sync per step; per step: one pinned-host -> device copy of the "
                                  "inputs, the three library calls, one device -> pinned-host copy of the output, replayed "
@@ -378,17 +382,21 @@ def run_ours(args):
         assert torch.equal(outs_h[0].view(torch.int16), out_eager.view(torch.int16)), "pipelined step and eager step disagree"
         assert torch.equal(outs_h[1].view(torch.int16), out_eager.view(torch.int16)), "pipelined step and eager step disagree"
         assert torch.equal(pool.k_pool, k0), "pool state drifted across pipelined steps"
+        dt_p, p_bytes = aggregate_over_ranks(dt_p * 1e3, float(step_bytes), dev)
+        dt_p *= 1e-3
         result["e2e"]["two_steps_in_flight"] = {
-            "value": round(step_bytes * world / dt_p / 1e9, 1), "ms_per_step": round(dt_p * 1e3, 5), "steps": Ke,
+            "value": round(p_bytes / dt_p / 1e9, 1), "ms_per_step": round(dt_p * 1e3, 5), "steps": Ke,
             "note": "same copies every step, on copy streams: step i + 1's upload and step i - 1's read-back overlap step i's "
                     "kernels; the host waits for a step's result two steps later"}
-        result["cpu_baseline"] = cpu_baseline(wl, tp_req, tp_idx, outs_d[0].to(torch.float64).cpu().numpy(), budget_s=20.0)
-        if not args.no_extras:
+        if rank == 0 and world == 1:                       # the oracle on the host cores: rank 0 at N = 1 only
+            result["cpu_baseline"] = cpu_baseline(wl, tp_req, tp_idx, outs_d[0].to(torch.float64).cpu().numpy(), budget_s=20.0)
+        if rank == 0 and world == 1 and not args.no_extras:
             result["extras"] = extras(b, torch, dev, args)
             result["roofline"]["others"] = roofline_others(result["extras"], peak)
     if world > 1:
+        dist.barrier()
         dist.destroy_process_group()
-    return result
+    return result if rank == 0 else None
 
 
 def cpu_baseline(wl, tp_req, tp_idx, gpu_out, budget_s):
