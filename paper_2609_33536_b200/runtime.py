@@ -71,6 +71,38 @@ class ElasticRuntime:
                                     v[5] if len(v[5]) else None, self.boundaries, self.flags)
         return self.flags
 
+    def layout(self):
+        """(any BASE pair, any irregular request) of the live requests, from the controller's state: a
+        request is irregular when a TARGET pair lies between two of its BASE pairs (Sec. 3.2)."""
+        any_base = irregular = False
+        for r, n in self.lens.items():
+            if n <= 0:
+                continue
+            modes = [self.ctrl.pair_mode(r, p) == 1 for p in range(len(self.ctrl.block_table(r)) // 2)]
+            if any(modes):
+                any_base = True
+                first, last = modes.index(True), len(modes) - 1 - modes[::-1].index(True)
+                irregular = irregular or not all(modes[first:last + 1])
+        return any_base, irregular
+
+    def decode(self, q, out, num_q_heads, sm_scale, workspace, layer=0):
+        """Decode attention with the dispatch of Sec. 3.2, decided on the host (no device read): a batch
+        without BASE pairs takes the native path, a batch whose sequences are all regular the structured
+        path (boundaries from the sparse lowering), any other the general path. Returns the path's name."""
+        any_base, irregular = self.layout()
+        msl = max([n for n in self.lens.values()] + [0])
+        if any_base and not irregular:
+            self.lower()
+            b.ekv_attn_decode_structured(self.pool, layer, self.batch, self.boundaries, q, out, num_q_heads, sm_scale, msl,
+                                         workspace)
+            return "structured"
+        self.batch.has_base = any_base
+        try:
+            b.ekv_attn_decode(self.pool, layer, self.batch, q, out, num_q_heads, sm_scale, msl, workspace)
+        finally:
+            self.batch.has_base = True
+        return "general" if any_base else "native"
+
     def add_request(self, req, n_tokens):
         self.ctrl.add_request(req, n_tokens)
         self.rows[req] = self.free_rows.pop()

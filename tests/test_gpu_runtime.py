@@ -38,6 +38,7 @@ def test_pressure_loop_with_controller(oracle):
     q = torch.from_numpy(q_bits.view(np.int16)).cuda().view(torch.bfloat16)
     out = torch.empty_like(q)
     saw_demotion = saw_promotion = False
+    paths = set()
     released_pairs = 0
     for step in range(14):
         # pressure for the first steps, then calm: the reserve decays and promotion gets a budget
@@ -69,6 +70,10 @@ def test_pressure_loop_with_controller(oracle):
         msl = int(max(lens))
         ws = b.new_workspace(pool, n_req, Hq, msl)
         b.ekv_attn_decode(pool, 0, rt.batch, q, out, Hq, D ** -0.5, msl, ws)
+        out2 = torch.empty_like(out)                                    # the runtime's own dispatch: native / structured / general
+        path = rt.decode(q, out2, Hq, D ** -0.5, ws)
+        paths.add(path)
+        assert torch.equal(out2.view(torch.int16), out.view(torch.int16)), f"step {step}: {path} path differs from the general one"
         prow, ppi, pnb, psl = rt.restore(transfer_slack=3)
         torch.cuda.synchronize()
         exp = oracle.attn_decode(op, 0, q_bits, Hq, D ** -0.5)          # attention ran before the promotion
@@ -89,6 +94,7 @@ def test_pressure_loop_with_controller(oracle):
             t = rt.ctrl.block_table(r)
             assert np.array_equal(t, rt.block_table[r, : len(t)].cpu().numpy())
     assert saw_demotion and saw_promotion
+    assert "native" in paths and len(paths) >= 2, paths
     assert rt.stats["demoted"] - rt.stats["promoted"] - released_pairs == rt.ctrl.base_pairs == int(pool.tags.sum().item())
 
 
