@@ -234,165 +234,165 @@ def run_ours(args):
     main_ms = float(np.mean([e0.elapsed_time(e1) for e0, e1 in prof]))
 
     result = None
-    if True:                                                # every rank: the end-to-end leg is measured on all of them
-        assert torch.equal(pool.k_pool, k0), "pool state drifted across steps"
-        clocks = sampler.stop() if sampler else None
-        peak, peak_src = _peaks()
-        achieved = kv_bytes / (main_ms * 1e-3) / 1e9
-        result = {
-            "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": K,
-            "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": WORKLOAD if args.batch == 64 else WORKLOAD.replace("batch 64", f"batch {args.batch}"), "seed": seed, "l2": "inputs larger than L2 (0.9 GB of KV per step vs 126 MB)",
-                       "tokens": int(wl.seq_lens.sum()), "realised_base_fraction": round(wl.realised_base_fraction(), 4),
-                       "bytes_per_step": int(step_bytes), "kv_bytes_per_step": int(kv_bytes),
-                       "multi_gpu": "replicas only (no exchange step on this path)"},
-            "clocks": clocks,
-            "gpu_launches": 4 * K,          # per step: downgrade pack, decode split, decode merge, refine expand
-            "roofline": {"bound": "hbm", "kernel": "decode_ring_kernel<128,true> (split kernel of ekv_attn_decode)",
-                         "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4),
-                         "frac_of_8000_nominal": round(achieved / 8000.0, 4), "peak_source": peak_src,
-                         "us_per_launch": round(main_ms * 1e3, 2), "launches_timed": n_prof,
-                         "traffic": round(kv_bytes * NCU_TRAFFIC_PER_KV_BYTE) if NCU_TRAFFIC_PER_KV_BYTE else None,
-                         "traffic_note": "dram read+write bytes of one ncu capture of this kernel on a smaller batch "
-                                         "of the same workload, scaled by the K/V bytes of a full launch"},
-            "tokens_per_s": round(wl.batch / (ms_per_step * 1e-3), 1),
-        }
-        if args.profile_only:
-            result["config"]["note"] = "profiling run: reduced batch, no e2e / cpu_baseline / extras"
-            return result if rank == 0 else None
-        # ---- end to end: host buffers, H2D of the step's inputs and D2H of its result, every step ----
-        # The step's inputs (queries, block table, sequence lengths, the transition batch) sit in ONE pinned
-        # host arena and travel in one copy to a device arena the calls read through views; the result comes
-        # back into pinned memory. Copy in, the three library calls and copy out are captured once as a CUDA
-        # graph on the caller's side (the library allocates nothing and orders everything on the stream it is
-        # given, so its calls can be captured as they are) and replayed once per step.
-        parts = [("q", wl.q.view(np.int16)), ("bt", batch.block_table.cpu().numpy()), ("sl", wl.seq_lens),
-                 ("req", tp_req), ("idx", tp_idx), ("slot", np.arange(n_tp, dtype=np.int32))]
-        offs, total = {}, 0
-        for name, a in parts:
-            offs[name] = total
-            total += (a.nbytes + 255) // 256 * 256
-        arena_h = torch.empty(total, dtype=torch.uint8).pin_memory()
-        arena_d = torch.empty(total, dtype=torch.uint8, device=dev)
-        for name, a in parts:
-            arena_h[offs[name]:offs[name] + a.nbytes].copy_(torch.from_numpy(np.ascontiguousarray(a)).view(torch.uint8).reshape(-1))
+    # every rank from here on: the end-to-end leg is measured on all of them
+    assert torch.equal(pool.k_pool, k0), "pool state drifted across steps"
+    clocks = sampler.stop() if sampler else None
+    peak, peak_src = _peaks()
+    achieved = kv_bytes / (main_ms * 1e-3) / 1e9
+    result = {
+        "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": K,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD if args.batch == 64 else WORKLOAD.replace("batch 64", f"batch {args.batch}"), "seed": seed, "l2": "inputs larger than L2 (0.9 GB of KV per step vs 126 MB)",
+                   "tokens": int(wl.seq_lens.sum()), "realised_base_fraction": round(wl.realised_base_fraction(), 4),
+                   "bytes_per_step": int(step_bytes), "kv_bytes_per_step": int(kv_bytes),
+                   "multi_gpu": "replicas only (no exchange step on this path)"},
+        "clocks": clocks,
+        "gpu_launches": 4 * K,          # per step: downgrade pack, decode split, decode merge, refine expand
+        "roofline": {"bound": "hbm", "kernel": "decode_ring_kernel<128,true> (split kernel of ekv_attn_decode)",
+                     "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4),
+                     "frac_of_8000_nominal": round(achieved / 8000.0, 4), "peak_source": peak_src,
+                     "us_per_launch": round(main_ms * 1e3, 2), "launches_timed": n_prof,
+                     "traffic": round(kv_bytes * NCU_TRAFFIC_PER_KV_BYTE) if NCU_TRAFFIC_PER_KV_BYTE else None,
+                     "traffic_note": "dram read+write bytes of one ncu capture of this kernel on a smaller batch "
+                                     "of the same workload, scaled by the K/V bytes of a full launch"},
+        "tokens_per_s": round(wl.batch / (ms_per_step * 1e-3), 1),
+    }
+    if args.profile_only:
+        result["config"]["note"] = "profiling run: reduced batch, no e2e / cpu_baseline / extras"
+        return result if rank == 0 else None
+    # ---- end to end: host buffers, H2D of the step's inputs and D2H of its result, every step ----
+    # The step's inputs (queries, block table, sequence lengths, the transition batch) sit in ONE pinned
+    # host arena and travel in one copy to a device arena the calls read through views; the result comes
+    # back into pinned memory. Copy in, the three library calls and copy out are captured once as a CUDA
+    # graph on the caller's side (the library allocates nothing and orders everything on the stream it is
+    # given, so its calls can be captured as they are) and replayed once per step.
+    parts = [("q", wl.q.view(np.int16)), ("bt", batch.block_table.cpu().numpy()), ("sl", wl.seq_lens),
+             ("req", tp_req), ("idx", tp_idx), ("slot", np.arange(n_tp, dtype=np.int32))]
+    offs, total = {}, 0
+    for name, a in parts:
+        offs[name] = total
+        total += (a.nbytes + 255) // 256 * 256
+    arena_h = torch.empty(total, dtype=torch.uint8).pin_memory()
+    arena_d = torch.empty(total, dtype=torch.uint8, device=dev)
+    for name, a in parts:
+        arena_h[offs[name]:offs[name] + a.nbytes].copy_(torch.from_numpy(np.ascontiguousarray(a)).view(torch.uint8).reshape(-1))
 
-        def dview(name, a, dtype):
-            return arena_d[offs[name]:offs[name] + a.nbytes].view(dtype).reshape(a.shape)
-        q2 = dview("q", wl.q, q.dtype)
-        batch2 = b.Batch(dview("bt", wl.block_table, torch.int32), dview("sl", wl.seq_lens, torch.int32), True)
-        req2, idx2, slot2 = (dview(n, tp_req, torch.int32) for n in ("req", "idx", "slot"))
-        outh = torch.empty(out.shape, dtype=out.dtype).pin_memory()
-        h2d, d2h = int(sum(a.nbytes for _, a in parts)), outh.numel() * 2
+    def dview(name, a, dtype):
+        return arena_d[offs[name]:offs[name] + a.nbytes].view(dtype).reshape(a.shape)
+    q2 = dview("q", wl.q, q.dtype)
+    batch2 = b.Batch(dview("bt", wl.block_table, torch.int32), dview("sl", wl.seq_lens, torch.int32), True)
+    req2, idx2, slot2 = (dview(n, tp_req, torch.int32) for n in ("req", "idx", "slot"))
+    outh = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+    h2d, d2h = int(sum(a.nbytes for _, a in parts)), outh.numel() * 2
 
-        def e2e_body():
-            arena_d.copy_(arena_h, non_blocking=True)
-            b.ekv_downgrade(pool, batch2, req2, idx2, kres, vres, slot2, freed)
-            b.ekv_attn_decode(pool, 0, batch2, q2, out, wl.num_q_heads, wl.sm_scale, msl, ws)
-            b.ekv_refine(pool, batch2, req2, idx2, freed, kres, vres, slot2)
-            outh.copy_(out, non_blocking=True)
+    def e2e_body():
+        arena_d.copy_(arena_h, non_blocking=True)
+        b.ekv_downgrade(pool, batch2, req2, idx2, kres, vres, slot2, freed)
+        b.ekv_attn_decode(pool, 0, batch2, q2, out, wl.num_q_heads, wl.sm_scale, msl, ws)
+        b.ekv_refine(pool, batch2, req2, idx2, freed, kres, vres, slot2)
+        outh.copy_(out, non_blocking=True)
 
-        def timed_e2e(fn, n):
-            for _ in range(3):
-                fn()
-            t0 = time.perf_counter()
-            for _ in range(n):
-                fn()
-            return (time.perf_counter() - t0) / n
-
-        def eager_step():
-            e2e_body()
-            torch.cuda.synchronize()
-
-        Ke = min(K, 500)
-        dt_eager = timed_e2e(eager_step, Ke)
-        out_eager = outh.clone()
-        side = torch.cuda.Stream()
-        side.wait_stream(torch.cuda.current_stream())
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(side):
-            e2e_body()                                       # warm the side stream before capture
-            side.synchronize()
-            with torch.cuda.graph(graph, stream=side):
-                e2e_body()
-        torch.cuda.synchronize()
-        outh.zero_()
-
-        def graph_step():
-            graph.replay()
-            torch.cuda.synchronize()
-
-        dt = timed_e2e(graph_step, Ke)
-        assert torch.equal(outh.view(torch.int16), out_eager.view(torch.int16)), "graph replay and eager step disagree"
-        assert torch.equal(pool.k_pool, k0), "pool state drifted across end-to-end steps"
-        # every rank measured its own replica: the job's time is the slowest rank's, its work the sum
-        dt, e2e_bytes = aggregate_over_ranks(dt * 1e3, float(step_bytes), dev)
-        dt *= 1e-3
-        dt_eager = aggregate_over_ranks(dt_eager * 1e3, 0.0, dev)[0] * 1e-3
-        result["e2e"] = {"value": round(e2e_bytes / dt / 1e9, 1), "unit": UNIT, "h2d_bytes_per_step": h2d * world,
-                         "d2h_bytes_per_step": int(d2h) * world, "ms_per_step": round(dt * 1e3, 5), "steps": Ke,
-                         "eager_ms_per_step": round(dt_eager * 1e3, 5),
-                         "note": "host wall clock, one stream sync per step; per step: one pinned-host -> device copy of the "
-                                 "inputs, the three library calls, one device -> pinned-host copy of the output, replayed "
-                                 "as one CUDA graph (eager_ms_per_step: the same sequence issued call by call); the KV pool "
-                                 "is resident cache state"}
-        # Two steps in flight: step i + 1's inputs go up on a copy stream and step i - 1's output comes down on
-        # another while step i's kernels run. Every step still uploads its own inputs from pinned memory and has
-        # its result read back to pinned memory; only the waiting is overlapped. Reported beside the serial figure.
-        arenas = [arena_d, torch.empty_like(arena_d)]
-        outs_d = [out, torch.empty_like(out)]
-        outs_h = [outh, torch.empty(out.shape, dtype=out.dtype).pin_memory()]
-        views = []
-        for a in arenas:
-            dv = lambda name, arr, dtype, a=a: a[offs[name]:offs[name] + arr.nbytes].view(dtype).reshape(arr.shape)
-            views.append((dv("q", wl.q, q.dtype), b.Batch(dv("bt", wl.block_table, torch.int32), dv("sl", wl.seq_lens, torch.int32), True),
-                          dv("req", tp_req, torch.int32), dv("idx", tp_idx, torch.int32), dv("slot", tp_req, torch.int32)))
-        s_in, s_out, s_main = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.current_stream()
-        ev_in = [torch.cuda.Event() for _ in range(2)]
-        ev_done = [torch.cuda.Event() for _ in range(2)]
-        ev_out = [torch.cuda.Event() for _ in range(2)]
-
-        def pipelined(n):
-            for i in range(n):
-                par = i & 1
-                if i >= 2:
-                    ev_out[par].synchronize()              # the host has step i - 2's result; its buffers are free again
-                with torch.cuda.stream(s_in):
-                    s_in.wait_event(ev_done[par])          # step i - 2 no longer reads this arena
-                    arenas[par].copy_(arena_h, non_blocking=True)
-                    ev_in[par].record()
-                s_main.wait_event(ev_in[par])
-                s_main.wait_event(ev_out[par])             # step i - 2's output has left outs_d[par]
-                q_v, batch_v, req_v, idx_v, slot_v = views[par]
-                b.ekv_downgrade(pool, batch_v, req_v, idx_v, kres, vres, slot_v, freed)
-                b.ekv_attn_decode(pool, 0, batch_v, q_v, outs_d[par], wl.num_q_heads, wl.sm_scale, msl, ws)
-                b.ekv_refine(pool, batch_v, req_v, idx_v, freed, kres, vres, slot_v)
-                ev_done[par].record()
-                with torch.cuda.stream(s_out):
-                    s_out.wait_event(ev_done[par])
-                    outs_h[par].copy_(outs_d[par], non_blocking=True)
-                    ev_out[par].record()
-            torch.cuda.synchronize()
-
-        pipelined(8)
+    def timed_e2e(fn, n):
+        for _ in range(3):
+            fn()
         t0 = time.perf_counter()
-        pipelined(Ke)
-        dt_p = (time.perf_counter() - t0) / Ke
-        assert torch.equal(outs_h[0].view(torch.int16), out_eager.view(torch.int16)), "pipelined step and eager step disagree"
-        assert torch.equal(outs_h[1].view(torch.int16), out_eager.view(torch.int16)), "pipelined step and eager step disagree"
-        assert torch.equal(pool.k_pool, k0), "pool state drifted across pipelined steps"
-        dt_p, p_bytes = aggregate_over_ranks(dt_p * 1e3, float(step_bytes), dev)
-        dt_p *= 1e-3
-        result["e2e"]["two_steps_in_flight"] = {
-            "value": round(p_bytes / dt_p / 1e9, 1), "ms_per_step": round(dt_p * 1e3, 5), "steps": Ke,
-            "note": "same copies every step, on copy streams: step i + 1's upload and step i - 1's read-back overlap step i's "
-                    "kernels; the host waits for a step's result two steps later"}
-        if rank == 0 and world == 1:                       # the oracle on the host cores: rank 0 at N = 1 only
-            result["cpu_baseline"] = cpu_baseline(wl, tp_req, tp_idx, outs_d[0].to(torch.float64).cpu().numpy(), budget_s=20.0)
-        if rank == 0 and world == 1 and not args.no_extras:
-            result["extras"] = extras(b, torch, dev, args)
-            result["roofline"]["others"] = roofline_others(result["extras"], peak)
+        for _ in range(n):
+            fn()
+        return (time.perf_counter() - t0) / n
+
+    def eager_step():
+        e2e_body()
+        torch.cuda.synchronize()
+
+    Ke = min(K, 500)
+    dt_eager = timed_e2e(eager_step, Ke)
+    out_eager = outh.clone()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        e2e_body()                                       # warm the side stream before capture
+        side.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            e2e_body()
+    torch.cuda.synchronize()
+    outh.zero_()
+
+    def graph_step():
+        graph.replay()
+        torch.cuda.synchronize()
+
+    dt = timed_e2e(graph_step, Ke)
+    assert torch.equal(outh.view(torch.int16), out_eager.view(torch.int16)), "graph replay and eager step disagree"
+    assert torch.equal(pool.k_pool, k0), "pool state drifted across end-to-end steps"
+    # every rank measured its own replica: the job's time is the slowest rank's, its work the sum
+    dt, e2e_bytes = aggregate_over_ranks(dt * 1e3, float(step_bytes), dev)
+    dt *= 1e-3
+    dt_eager = aggregate_over_ranks(dt_eager * 1e3, 0.0, dev)[0] * 1e-3
+    result["e2e"] = {"value": round(e2e_bytes / dt / 1e9, 1), "unit": UNIT, "h2d_bytes_per_step": h2d * world,
+                     "d2h_bytes_per_step": int(d2h) * world, "ms_per_step": round(dt * 1e3, 5), "steps": Ke,
+                     "eager_ms_per_step": round(dt_eager * 1e3, 5),
+                     "note": "host wall clock, one stream sync per step; per step: one pinned-host -> device copy of the "
+                             "inputs, the three library calls, one device -> pinned-host copy of the output, replayed "
+                             "as one CUDA graph (eager_ms_per_step: the same sequence issued call by call); the KV pool "
+                             "is resident cache state"}
+    # Two steps in flight: step i + 1's inputs go up on a copy stream and step i - 1's output comes down on
+    # another while step i's kernels run. Every step still uploads its own inputs from pinned memory and has
+    # its result read back to pinned memory; only the waiting is overlapped. Reported beside the serial figure.
+    arenas = [arena_d, torch.empty_like(arena_d)]
+    outs_d = [out, torch.empty_like(out)]
+    outs_h = [outh, torch.empty(out.shape, dtype=out.dtype).pin_memory()]
+    views = []
+    for a in arenas:
+        dv = lambda name, arr, dtype, a=a: a[offs[name]:offs[name] + arr.nbytes].view(dtype).reshape(arr.shape)
+        views.append((dv("q", wl.q, q.dtype), b.Batch(dv("bt", wl.block_table, torch.int32), dv("sl", wl.seq_lens, torch.int32), True),
+                      dv("req", tp_req, torch.int32), dv("idx", tp_idx, torch.int32), dv("slot", tp_req, torch.int32)))
+    s_in, s_out, s_main = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.current_stream()
+    ev_in = [torch.cuda.Event() for _ in range(2)]
+    ev_done = [torch.cuda.Event() for _ in range(2)]
+    ev_out = [torch.cuda.Event() for _ in range(2)]
+
+    def pipelined(n):
+        for i in range(n):
+            par = i & 1
+            if i >= 2:
+                ev_out[par].synchronize()              # the host has step i - 2's result; its buffers are free again
+            with torch.cuda.stream(s_in):
+                s_in.wait_event(ev_done[par])          # step i - 2 no longer reads this arena
+                arenas[par].copy_(arena_h, non_blocking=True)
+                ev_in[par].record()
+            s_main.wait_event(ev_in[par])
+            s_main.wait_event(ev_out[par])             # step i - 2's output has left outs_d[par]
+            q_v, batch_v, req_v, idx_v, slot_v = views[par]
+            b.ekv_downgrade(pool, batch_v, req_v, idx_v, kres, vres, slot_v, freed)
+            b.ekv_attn_decode(pool, 0, batch_v, q_v, outs_d[par], wl.num_q_heads, wl.sm_scale, msl, ws)
+            b.ekv_refine(pool, batch_v, req_v, idx_v, freed, kres, vres, slot_v)
+            ev_done[par].record()
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_done[par])
+                outs_h[par].copy_(outs_d[par], non_blocking=True)
+                ev_out[par].record()
+        torch.cuda.synchronize()
+
+    pipelined(8)
+    t0 = time.perf_counter()
+    pipelined(Ke)
+    dt_p = (time.perf_counter() - t0) / Ke
+    assert torch.equal(outs_h[0].view(torch.int16), out_eager.view(torch.int16)), "pipelined step and eager step disagree"
+    assert torch.equal(outs_h[1].view(torch.int16), out_eager.view(torch.int16)), "pipelined step and eager step disagree"
+    assert torch.equal(pool.k_pool, k0), "pool state drifted across pipelined steps"
+    dt_p, p_bytes = aggregate_over_ranks(dt_p * 1e3, float(step_bytes), dev)
+    dt_p *= 1e-3
+    result["e2e"]["two_steps_in_flight"] = {
+        "value": round(p_bytes / dt_p / 1e9, 1), "ms_per_step": round(dt_p * 1e3, 5), "steps": Ke,
+        "note": "same copies every step, on copy streams: step i + 1's upload and step i - 1's read-back overlap step i's "
+                "kernels; the host waits for a step's result two steps later"}
+    if rank == 0 and world == 1:                       # the oracle on the host cores: rank 0 at N = 1 only
+        result["cpu_baseline"] = cpu_baseline(wl, tp_req, tp_idx, outs_d[0].to(torch.float64).cpu().numpy(), budget_s=20.0)
+    if rank == 0 and world == 1 and not args.no_extras:
+        result["extras"] = extras(b, torch, dev, args)
+        result["roofline"]["others"] = roofline_others(result["extras"], peak)
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
